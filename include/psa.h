@@ -1,0 +1,142 @@
+/*
+ * psa.h -- C interface of libpsa: skip-scheduled single-layer multi-head self-attention for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library computes, per (batch item, head), the three phases of self-attention
+ *     phase 1  S_ij = scale * sum_c q_i[c] k_j[c]                 (paper Eq. 1; scale = 1/sqrt(d_k))
+ *     phase 2  w_ij = exp(S_ij) / sum_j exp(S_ij)                 (paper Eq. 2)
+ *     phase 3  y_i  = sum_j w_ij v_j                              (paper Eq. 3)
+ * optionally preceded by the projections q,k,v = x*Wq, x*Wk, x*Wv (paper Sec. 3.1), under one of
+ * three schemes that decide which weights are ever issued (never "computed, then masked"):
+ *     PSA_FULL       the original definition (paper Sec. 3.2)
+ *     PSA_SYMMETRIC  query = key = value: one member of each pair (S_ij, S_ji) is computed in
+ *                    phase 1 and reused for the other; phases 2 and 3 are unchanged (paper Sec. 4)
+ *     PSA_MASKED     decoder mask: only weights with j <= i take part, in all phases (paper Sec. 5)
+ *
+ * General conventions
+ *   - Unless an entry point says "host", every data pointer is a DEVICE pointer owned by the
+ *     caller.  The library neither frees nor keeps it after the call returns, except the workspace
+ *     registered with psa_set_workspace.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls enqueue
+ *     work on it and return without waiting; argument errors are reported immediately and launch
+ *     nothing.  Conditions only the device can see (a bounded wait that expired) are recorded in a
+ *     device status word and reported by psa_last_issued.
+ *   - All tensors are dense, row-major, 16-byte aligned:
+ *         X    [batch, n, d_model]
+ *         W*   [d_model, heads*d_k]      head h owns columns h*d_k .. (h+1)*d_k-1
+ *         Q,K,V[batch, n, heads, d_k]
+ *         out  [batch, n, heads*d_k]
+ *   - Every function returns a psa_status (0 = PSA_OK) unless stated otherwise.
+ *   - Calls that share a workspace must be ordered on one stream; the library is not re-entrant
+ *     across streams.
+ */
+#ifndef PSA_H_
+#define PSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { PSA_FULL = 0, PSA_SYMMETRIC = 1, PSA_MASKED = 2 } psa_scheme;
+typedef enum { PSA_F32 = 0, PSA_BF16 = 1 } psa_dtype;
+
+typedef enum {
+    PSA_OK = 0,
+    PSA_ERR_NULL = 1,        /* a required pointer is NULL                                     */
+    PSA_ERR_SHAPE = 2,       /* a size is <= 0 or overflows                                    */
+    PSA_ERR_UNSUPPORTED = 3, /* shape outside what the kernels cover (see each entry point)     */
+    PSA_ERR_ALIGN = 4,       /* a pointer is not 16-byte aligned                               */
+    PSA_ERR_SCHEME_ARGS = 5, /* unknown scheme, or PSA_SYMMETRIC given distinct k/v operands   */
+    PSA_ERR_WORKSPACE = 6,   /* registered workspace too small and growing it failed           */
+    PSA_ERR_CUDA = 7,        /* a CUDA runtime/driver call failed (psa_last_cuda_error)        */
+    PSA_ERR_TIMEOUT = 8,     /* a bounded device-side wait expired; results are invalid        */
+    PSA_ERR_NUMERIC = 9      /* reserved                                                       */
+} psa_status;
+
+/*
+ * Multiply-accumulate census of one call (summed over batch and heads).
+ *   proj_macs       projection MACs (paper Sec. 3.1; not part of the paper's own count)
+ *   qk_macs         phase-1 MACs issued      pv_macs   phase-3 MACs issued
+ *   exps            phase-2 exponentials evaluated
+ *   useful_*        the paper's element-level counts for the scheme (Sec. 3.2, 4.2, 5.2):
+ *                   FULL d*n^2 each; MASKED d*n(n+1)/2 each; SYMMETRIC d*n(n+1)/2 and d*n^2
+ * The bf16 path issues whole 128x128 blocks of the weight matrix, so issued >= useful there (a
+ * block on the diagonal is issued in full); the fp32 path skips element by element, issued = useful.
+ */
+typedef struct {
+    uint64_t proj_macs, qk_macs, pv_macs, exps, useful_qk_macs, useful_pv_macs;
+} psa_counts;
+
+/*
+ * Projections + attention, bf16 in / bf16 out, fp32 accumulation (paper Sec. 3.1 then Eq. 1-3).
+ *   X, Wq, Wk, Wv, out   device, bf16, layouts above.
+ *   PSA_SYMMETRIC: q = k = v = X*Wq (paper Sec. 4.1); Wk and Wv must be NULL or equal to Wq.
+ * Supported: d_k in {64, 128}; n a multiple of 128; d_model and heads*d_k multiples of 64.
+ * Needs a workspace of psa_workspace_bytes(...) (grown on demand, see psa_set_workspace).
+ */
+int psa_attention(const void* X, const void* Wq, const void* Wk, const void* Wv, int batch, int heads, int n,
+                  int d_model, int d_k, int scheme, void* out, void* stream);
+
+/* Same computation in fp32 storage and fp32 arithmetic on CUDA cores, element-exact skipping
+ * (issued = useful).  Supported: n <= 1024, d_k <= 128 (any d_model). */
+int psa_attention_f32(const void* X, const void* Wq, const void* Wk, const void* Wv, int batch, int heads, int n,
+                      int d_model, int d_k, int scheme, void* out, void* stream);
+
+/*
+ * Attention core only (paper Eq. 1-3 with q, k, v given; Sec. 3.1 last paragraph).
+ *   dtype PSA_BF16 or PSA_F32 selects the path and the storage type of Q, K, V, out.
+ *   PSA_SYMMETRIC: K and V must be NULL or equal to Q.
+ * Shape limits as for psa_attention / psa_attention_f32.
+ */
+int psa_attention_core(const void* Q, const void* K, const void* V, int batch, int heads, int n, int d_k,
+                       int scheme, int dtype, void* out, void* stream);
+
+/*
+ * psa_attention / psa_attention_f32 with HOST buffers (pageable or pinned): copies X and the
+ * projection matrices to the device, runs the layer, copies `out` back and waits for `stream`.
+ * dtype selects bf16 or fp32 storage.  The staging buffers are part of the workspace.
+ */
+int psa_attention_host(const void* X_host, const void* Wq_host, const void* Wk_host, const void* Wv_host,
+                       int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, void* out_host,
+                       void* stream);
+
+/*
+ * Analytic census: what the tile scheduler will issue for this shape and scheme (paper Sec. 3.2,
+ * 4.2, 5.2 for the useful_* fields).  Host only, launches nothing.  d_model = 0 means "core only"
+ * (proj_macs = 0).
+ */
+int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, psa_counts* counts);
+
+/*
+ * Measured census: waits for `stream`, then returns the counters the kernels of the last call
+ * accumulated on the device (one increment per block of work actually issued) and that call's
+ * device status (PSA_OK or PSA_ERR_TIMEOUT).
+ */
+int psa_last_issued(void* stream, psa_counts* counts);
+
+/* Bytes of scratch memory a call with these arguments needs (projected q, k, v; the symmetric
+ * scheme's score matrix; counters).  with_host_staging != 0 adds psa_attention_host's buffers. */
+size_t psa_workspace_bytes(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype,
+                           int with_host_staging);
+
+/*
+ * Registers caller-owned device memory (256-byte aligned) as the workspace; it must stay valid
+ * until replaced or until psa_set_workspace(NULL, 0).  Without a registered workspace, or when it
+ * is too small, the library keeps a private one and grows it with cudaMalloc (synchronously, on
+ * the first call that needs more).
+ */
+int psa_set_workspace(void* dev_ptr, size_t bytes);
+
+/* Text for a psa_status; never NULL. */
+const char* psa_status_string(int status);
+
+/* Text of the last CUDA error seen by the calling thread's most recent failing call ("" if none). */
+const char* psa_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSA_H_ */

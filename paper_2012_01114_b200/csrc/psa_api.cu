@@ -1,0 +1,343 @@
+// C interface of libpsa: argument checking, workspace management, the host twin of the tile
+// scheduler (psa_skip_count) and dispatch to the fp32 and bf16 kernel families.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "psa_internal.h"
+#include "psa_sched.h"
+
+namespace psa {
+
+namespace {
+
+thread_local char g_err_text[256] = "";
+
+struct Context {
+    std::mutex mu;
+    void* user_ws = nullptr;
+    size_t user_bytes = 0;
+    void* own_ws = nullptr;
+    size_t own_bytes = 0;
+    int own_device = -1;
+    DeviceCounters* last_dc = nullptr;  // counters of the most recent call
+    psa_counts last_useful = {0, 0, 0, 0, 0, 0};
+};
+Context g_ctx;
+
+constexpr size_t COUNTER_BYTES = 256;
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, bool with_proj) {
+    if (scheme != PSA_FULL && scheme != PSA_SYMMETRIC && scheme != PSA_MASKED) return PSA_ERR_SCHEME_ARGS;
+    if (dtype != PSA_F32 && dtype != PSA_BF16) return PSA_ERR_UNSUPPORTED;
+    if (batch <= 0 || heads <= 0 || n <= 0 || d_k <= 0 || (with_proj && d_model <= 0)) return PSA_ERR_SHAPE;
+    if ((double)batch * heads * n * (double)d_k > 4.0e12 || (double)batch * n * (double)(with_proj ? d_model : 1) > 4.0e12)
+        return PSA_ERR_SHAPE;
+    if ((long long)batch * n > 0x7fffffffLL || (long long)heads * d_k > 0x7fffffffLL) return PSA_ERR_SHAPE;
+    if (dtype == PSA_BF16) {
+        if (d_k != 64 && d_k != 128) return PSA_ERR_UNSUPPORTED;
+        if (n % TILE != 0) return PSA_ERR_UNSUPPORTED;
+        if (with_proj && (d_model % 64 != 0)) return PSA_ERR_UNSUPPORTED;
+    } else {
+        if (n > 1024 || d_k > 128) return PSA_ERR_UNSUPPORTED;
+    }
+    return PSA_OK;
+}
+
+struct WsLayout {
+    size_t q, k, v, s, s_bytes, xs, wq, wk, wv, outs, total;
+};
+
+WsLayout ws_layout(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, bool with_proj,
+                   bool staging) {
+    const size_t es = dtype == PSA_BF16 ? 2 : 4;
+    const size_t qkv = align_up((size_t)batch * n * heads * d_k * es, 256);
+    WsLayout L;
+    memset(&L, 0, sizeof(L));
+    size_t off = COUNTER_BYTES;
+    if (with_proj) {
+        L.q = off; off += qkv;
+        if (scheme == PSA_SYMMETRIC) { L.k = L.q; L.v = L.q; }
+        else { L.k = off; off += qkv; L.v = off; off += qkv; }
+    }
+    if (scheme == PSA_SYMMETRIC) {
+        L.s_bytes = dtype == PSA_BF16 ? bf16_symmetric_scratch_bytes(batch, heads, n)
+                                      : align_up((size_t)batch * heads * n * n * sizeof(float), 256);
+        L.s = off; off += L.s_bytes;
+    }
+    if (staging) {
+        const size_t xb = align_up((size_t)batch * n * d_model * es, 256);
+        const size_t wb = align_up((size_t)d_model * heads * d_k * es, 256);
+        L.xs = off; off += xb;
+        L.wq = off; off += wb;
+        if (scheme == PSA_SYMMETRIC) { L.wk = L.wq; L.wv = L.wq; }
+        else { L.wk = off; off += wb; L.wv = off; off += wb; }
+        L.outs = off; off += qkv;
+    }
+    L.total = off;
+    return L;
+}
+
+// Returns the base of a workspace of at least `bytes`, or nullptr (error text set).
+char* acquire_ws(size_t bytes) {
+    if (g_ctx.user_ws && g_ctx.user_bytes >= bytes) return static_cast<char*>(g_ctx.user_ws);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaGetDevice"); return nullptr; }
+    if (g_ctx.own_ws && g_ctx.own_device == dev && g_ctx.own_bytes >= bytes) return static_cast<char*>(g_ctx.own_ws);
+    if (g_ctx.own_ws) {
+        cudaDeviceSynchronize();
+        cudaFree(g_ctx.own_ws);
+        g_ctx.own_ws = nullptr;
+        g_ctx.own_bytes = 0;
+    }
+    void* p = nullptr;
+    e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaMalloc(workspace)"); return nullptr; }
+    g_ctx.own_ws = p;
+    g_ctx.own_bytes = bytes;
+    g_ctx.own_device = dev;
+    return static_cast<char*>(p);
+}
+
+void useful_counts(int batch, int heads, int n, int d_model, int d_k, int scheme, bool with_proj, psa_counts* c) {
+    const uint64_t bh = (uint64_t)batch * heads, N = n, d = d_k;
+    const uint64_t tri = N * (N + 1) / 2;
+    c->useful_qk_macs = bh * d * (scheme == PSA_FULL ? N * N : tri);
+    c->useful_pv_macs = bh * d * (scheme == PSA_MASKED ? tri : N * N);
+    const uint64_t nproj = scheme == PSA_SYMMETRIC ? 1 : 3;
+    c->proj_macs = with_proj ? nproj * (uint64_t)batch * N * (uint64_t)d_model * (uint64_t)heads * d : 0;
+}
+
+int run_layer(const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Q, const void* K,
+              const void* V, int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, void* out,
+              cudaStream_t stream, bool with_proj, char* ws, const WsLayout& L) {
+    DeviceCounters* dc = reinterpret_cast<DeviceCounters*>(ws);
+    cudaError_t e = cudaMemsetAsync(dc, 0, sizeof(DeviceCounters), stream);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaMemsetAsync(counters)"); return PSA_ERR_CUDA; }
+    g_ctx.last_dc = dc;
+    memset(&g_ctx.last_useful, 0, sizeof(psa_counts));
+    useful_counts(batch, heads, n, d_model, d_k, scheme, with_proj, &g_ctx.last_useful);
+    const float scale = 1.0f / sqrtf((float)d_k);
+    const int nW = scheme == PSA_SYMMETRIC ? 1 : 3;
+    if (with_proj) {
+        void* outs[3] = {ws + L.q, ws + L.k, ws + L.v};
+        const void* Ws[3] = {Wq, nW == 3 ? Wk : Wq, nW == 3 ? Wv : Wq};
+        if (dtype == PSA_F32) {
+            e = f32_project(static_cast<const float*>(X), reinterpret_cast<const float* const*>(Ws),
+                            reinterpret_cast<float* const*>(outs), nW, batch * n, d_model, heads * d_k, dc, stream);
+            if (e != cudaSuccess) { set_cuda_error(e, "f32_project"); return PSA_ERR_CUDA; }
+        } else {
+            int rc = bf16_project(X, Ws, outs, nW, batch * n, d_model, heads * d_k, dc, stream);
+            if (rc != PSA_OK) return rc;
+        }
+        Q = ws + L.q; K = ws + L.k; V = ws + L.v;
+    }
+    float* S = scheme == PSA_SYMMETRIC ? reinterpret_cast<float*>(ws + L.s) : nullptr;
+    if (dtype == PSA_F32) {
+        e = f32_attention(static_cast<const float*>(Q), static_cast<const float*>(K), static_cast<const float*>(V),
+                          static_cast<float*>(out), S, batch, heads, n, d_k, scale, scheme, dc, stream);
+        if (e != cudaSuccess) { set_cuda_error(e, "f32_attention"); return PSA_ERR_CUDA; }
+        return PSA_OK;
+    }
+    return bf16_attention(Q, K, V, out, S, L.s_bytes, batch, heads, n, d_k, scale, scheme, dc, stream);
+}
+
+int layer_entry(const void* X, const void* Wq, const void* Wk, const void* Wv, int batch, int heads, int n,
+                int d_model, int d_k, int scheme, int dtype, void* out, void* stream) {
+    g_err_text[0] = 0;
+    int rc = check_shape(batch, heads, n, d_model, d_k, scheme, dtype, true);
+    if (rc != PSA_OK) return rc;
+    if (!X || !Wq || !out) return PSA_ERR_NULL;
+    if (scheme == PSA_SYMMETRIC) {
+        if ((Wk && Wk != Wq) || (Wv && Wv != Wq)) return PSA_ERR_SCHEME_ARGS;
+    } else if (!Wk || !Wv) {
+        return PSA_ERR_NULL;
+    }
+    if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(out)) return PSA_ERR_ALIGN;
+    if (dtype == PSA_BF16 && (heads * d_k) % 64 != 0) return PSA_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    const WsLayout L = ws_layout(batch, heads, n, d_model, d_k, scheme, dtype, true, false);
+    char* ws = acquire_ws(L.total);
+    if (!ws) return PSA_ERR_WORKSPACE;
+    return run_layer(X, Wq, Wk, Wv, nullptr, nullptr, nullptr, batch, heads, n, d_model, d_k, scheme, dtype, out,
+                     static_cast<cudaStream_t>(stream), true, ws, L);
+}
+
+}  // namespace
+
+void set_cuda_error(cudaError_t e, const char* where) {
+    snprintf(g_err_text, sizeof(g_err_text), "%s: %s", where, cudaGetErrorString(e));
+}
+void set_error_text(const char* text) { snprintf(g_err_text, sizeof(g_err_text), "%s", text); }
+
+}  // namespace psa
+
+using namespace psa;
+
+extern "C" {
+
+int psa_attention(const void* X, const void* Wq, const void* Wk, const void* Wv, int batch, int heads, int n,
+                  int d_model, int d_k, int scheme, void* out, void* stream) {
+    return layer_entry(X, Wq, Wk, Wv, batch, heads, n, d_model, d_k, scheme, PSA_BF16, out, stream);
+}
+
+int psa_attention_f32(const void* X, const void* Wq, const void* Wk, const void* Wv, int batch, int heads, int n,
+                      int d_model, int d_k, int scheme, void* out, void* stream) {
+    return layer_entry(X, Wq, Wk, Wv, batch, heads, n, d_model, d_k, scheme, PSA_F32, out, stream);
+}
+
+int psa_attention_core(const void* Q, const void* K, const void* V, int batch, int heads, int n, int d_k,
+                       int scheme, int dtype, void* out, void* stream) {
+    g_err_text[0] = 0;
+    int rc = check_shape(batch, heads, n, 0, d_k, scheme, dtype, false);
+    if (rc != PSA_OK) return rc;
+    if (!Q || !out) return PSA_ERR_NULL;
+    if (scheme == PSA_SYMMETRIC) {
+        if ((K && K != Q) || (V && V != Q)) return PSA_ERR_SCHEME_ARGS;
+        K = Q; V = Q;
+    } else if (!K || !V) {
+        return PSA_ERR_NULL;
+    }
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(out)) return PSA_ERR_ALIGN;
+    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    const WsLayout L = ws_layout(batch, heads, n, 0, d_k, scheme, dtype, false, false);
+    char* ws = acquire_ws(L.total);
+    if (!ws) return PSA_ERR_WORKSPACE;
+    return run_layer(nullptr, nullptr, nullptr, nullptr, Q, K, V, batch, heads, n, 0, d_k, scheme, dtype, out,
+                     static_cast<cudaStream_t>(stream), false, ws, L);
+}
+
+int psa_attention_host(const void* X_host, const void* Wq_host, const void* Wk_host, const void* Wv_host,
+                       int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, void* out_host,
+                       void* stream_v) {
+    g_err_text[0] = 0;
+    int rc = check_shape(batch, heads, n, d_model, d_k, scheme, dtype, true);
+    if (rc != PSA_OK) return rc;
+    if (!X_host || !Wq_host || !out_host) return PSA_ERR_NULL;
+    if (scheme == PSA_SYMMETRIC) {
+        if ((Wk_host && Wk_host != Wq_host) || (Wv_host && Wv_host != Wq_host)) return PSA_ERR_SCHEME_ARGS;
+    } else if (!Wk_host || !Wv_host) {
+        return PSA_ERR_NULL;
+    }
+    if (dtype == PSA_BF16 && (heads * d_k) % 64 != 0) return PSA_ERR_UNSUPPORTED;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    const WsLayout L = ws_layout(batch, heads, n, d_model, d_k, scheme, dtype, true, true);
+    char* ws = acquire_ws(L.total);
+    if (!ws) return PSA_ERR_WORKSPACE;
+    const size_t es = dtype == PSA_BF16 ? 2 : 4;
+    const size_t xb = (size_t)batch * n * d_model * es, wb = (size_t)d_model * heads * d_k * es;
+    const size_t ob = (size_t)batch * n * heads * d_k * es;
+    cudaError_t e = cudaMemcpyAsync(ws + L.xs, X_host, xb, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ws + L.wq, Wq_host, wb, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess && scheme != PSA_SYMMETRIC) {
+        e = cudaMemcpyAsync(ws + L.wk, Wk_host, wb, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(ws + L.wv, Wv_host, wb, cudaMemcpyHostToDevice, stream);
+    }
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaMemcpyAsync(H2D)"); return PSA_ERR_CUDA; }
+    rc = run_layer(ws + L.xs, ws + L.wq, ws + L.wk, ws + L.wv, nullptr, nullptr, nullptr, batch, heads, n, d_model,
+                   d_k, scheme, dtype, ws + L.outs, stream, true, ws, L);
+    if (rc != PSA_OK) return rc;
+    e = cudaMemcpyAsync(out_host, ws + L.outs, ob, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaMemcpyAsync(D2H)/sync"); return PSA_ERR_CUDA; }
+    return PSA_OK;
+}
+
+int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, psa_counts* c) {
+    if (!c) return PSA_ERR_NULL;
+    const bool with_proj = d_model > 0;
+    int rc = check_shape(batch, heads, n, d_model, d_k, scheme, dtype, with_proj);
+    if (rc != PSA_OK) return rc;
+    memset(c, 0, sizeof(*c));
+    useful_counts(batch, heads, n, d_model, d_k, scheme, with_proj, c);
+    const uint64_t bh = (uint64_t)batch * heads;
+    if (dtype == PSA_F32) {  // element-exact skipping
+        c->qk_macs = c->useful_qk_macs;
+        c->pv_macs = c->useful_pv_macs;
+        c->exps = c->useful_pv_macs / (uint64_t)d_k;
+        return PSA_OK;
+    }
+    // bf16: walk the CTA list and each CTA's block list exactly as the kernels do.
+    const int T = row_tiles(n);
+    const uint64_t block_macs = (uint64_t)TILE * TILE * d_k;
+    uint64_t qk_blocks = 0, pv_blocks = 0;
+    const int P = ctas_per_head(n);
+    for (int cta = 0; cta < P; ++cta) {  // every head has the same list
+        const CtaWork w = cta_work(cta, n, scheme == PSA_MASKED);
+        for (int t = 0; t < w.ntiles; ++t) {
+            const int kv = kv_tiles(w.tile0 + t, T, scheme);
+            pv_blocks += kv;
+            if (scheme != PSA_SYMMETRIC) qk_blocks += kv;
+        }
+    }
+    if (scheme == PSA_SYMMETRIC) {
+        for (int t = 0; t < sym_pairs(T); ++t) {
+            int I, J;
+            sym_pair(t, &I, &J);
+            if (J <= I) ++qk_blocks;
+        }
+    }
+    c->qk_macs = bh * qk_blocks * block_macs;
+    c->pv_macs = bh * pv_blocks * block_macs;
+    c->exps = bh * pv_blocks * (uint64_t)TILE * TILE;
+    return PSA_OK;
+}
+
+int psa_last_issued(void* stream, psa_counts* c) {
+    if (!c) return PSA_ERR_NULL;
+    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    if (!g_ctx.last_dc) return PSA_ERR_NULL;
+    DeviceCounters h;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = cudaMemcpy(&h, g_ctx.last_dc, sizeof(h), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { set_cuda_error(e, "psa_last_issued"); return PSA_ERR_CUDA; }
+    *c = g_ctx.last_useful;
+    c->proj_macs = h.proj_macs;
+    c->qk_macs = h.qk_macs;
+    c->pv_macs = h.pv_macs;
+    c->exps = h.exps;
+    return h.status;
+}
+
+size_t psa_workspace_bytes(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype,
+                           int with_host_staging) {
+    const bool with_proj = d_model > 0;
+    if (check_shape(batch, heads, n, d_model, d_k, scheme, dtype, with_proj) != PSA_OK) return 0;
+    return ws_layout(batch, heads, n, d_model, d_k, scheme, dtype, with_proj, with_host_staging != 0 && with_proj).total;
+}
+
+int psa_set_workspace(void* dev_ptr, size_t bytes) {
+    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255u)) return PSA_ERR_ALIGN;
+    g_ctx.user_ws = dev_ptr;
+    g_ctx.user_bytes = dev_ptr ? bytes : 0;
+    g_ctx.last_dc = nullptr;
+    return PSA_OK;
+}
+
+const char* psa_status_string(int status) {
+    switch (status) {
+        case PSA_OK: return "ok";
+        case PSA_ERR_NULL: return "a required pointer is NULL";
+        case PSA_ERR_SHAPE: return "invalid size";
+        case PSA_ERR_UNSUPPORTED: return "shape or number type not supported by this path";
+        case PSA_ERR_ALIGN: return "pointer not sufficiently aligned";
+        case PSA_ERR_SCHEME_ARGS: return "unknown scheme, or operands inconsistent with the scheme";
+        case PSA_ERR_WORKSPACE: return "workspace unavailable";
+        case PSA_ERR_CUDA: return "CUDA call failed";
+        case PSA_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case PSA_ERR_NUMERIC: return "numeric failure";
+        default: return "unknown status";
+    }
+}
+
+const char* psa_last_cuda_error(void) { return g_err_text; }
+
+}  // extern "C"

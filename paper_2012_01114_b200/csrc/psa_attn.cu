@@ -1,0 +1,496 @@
+// Fused attention core for the bf16 path: phases 1-3 of the paper (Eq. 1-3) per (batch, head) and
+// per pair of 128-row query tiles, never materialising the n x n weight matrix.
+//
+//   phase 1  S = Q K^T            tcgen05 MMA, operands staged by TMA, accumulator in TMEM
+//   phase 2  softmax              one thread per query row reads its row of S from TMEM, keeps a
+//                                 running row maximum m and row sum l (the division of Eq. 2 is
+//                                 applied once to the output row), writes P = exp2(..) as bf16 back
+//                                 into TMEM over S
+//   phase 3  O += P V             tcgen05 MMA with P read from TMEM and V (row-major = MN-major) from
+//                                 shared memory, accumulator O in TMEM
+//
+// Which (row tile, column tile) blocks exist is decided by the tile scheduler (psa_sched.h): for
+// the masked scheme (paper Sec. 5) column tiles beyond the diagonal are absent from every loop in
+// this file -- not loaded, not multiplied, not exponentiated -- and only the block on the diagonal
+// carries an element predicate.  For the symmetric scheme (paper Sec. 4) phase 1 is a separate
+// kernel that computes one block per unordered tile pair and stores it at both mirror positions;
+// this kernel then runs phases 2 and 3 reading S from that scratch.
+//
+// CTA layout (384 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 4-7 = softmax and
+// epilogue of row tile 0, warps 8-11 = the same for row tile 1.  The two row tiles ping-pong: while
+// the softmax warps of one work on S_j, the tensor core runs the other's MMAs.
+// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [256+D,256+2D); P_t overlays S_t.
+#include "psa_internal.h"
+#include "psa_sched.h"
+#include "psa_tma.h"
+#include "sm100.cuh"
+
+namespace psa {
+
+namespace {
+
+constexpr int ATTN_THREADS = 384;
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float RESCALE_THRESHOLD = 8.0f;  // log2 units: O and l are rescaled only when the row max grew by more
+
+template <int D>
+struct AttnCfg {
+    static constexpr int SUB = D / 64;                  // 64-column sub-tiles per 128-row tile
+    static constexpr int TILE_BYTES = 128 * D * 2;      // one Q, K or V tile
+    static constexpr int KSTAGES = D == 128 ? 2 : 4;
+    static constexpr int VSTAGES = D == 128 ? 2 : 4;
+    static constexpr int SMEM = (2 + KSTAGES + VSTAGES) * TILE_BYTES + 1024;
+    static constexpr int TMEM_S = 0, TMEM_O = 256;
+};
+
+struct AttnMaps {
+    CUtensorMap q, k, v, o;
+};
+
+struct AttnBars {
+    uint64_t q_full[2];
+    uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
+    uint64_t s_full[2], p_ready[2], o_done[2];
+};
+
+template <int D, bool SYM>
+__global__ void __launch_bounds__(ATTN_THREADS, 1)
+attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg, int n, int H, int scheme, int bh0,
+            float sl2, DeviceCounters* dc) {
+    using Cfg = AttnCfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sQ = smem;                                          // 2 tiles
+    uint8_t* sK = sQ + 2 * Cfg::TILE_BYTES;                      // KSTAGES tiles
+    uint8_t* sV = sK + Cfg::KSTAGES * Cfg::TILE_BYTES;           // VSTAGES tiles
+    __shared__ AttnBars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int T = row_tiles(n);
+    const CtaWork work = cta_work(blockIdx.x, n, scheme == PSA_MASKED);
+    const int bh = bh0 + work.bh;
+    const int b = bh / H, h = bh - b * H;
+    const int row0 = b * n, col0 = h * D;
+    int nkv[2];
+    nkv[0] = kv_tiles(work.tile0, T, scheme);
+    nkv[1] = work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0;
+    const int maxkv = max(nkv[0], nkv[1]);
+    const int last_t = work.ntiles - 1;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&bars.q_full[t], 1);
+            mbar_init(&bars.s_full[t], 1);
+            mbar_init(&bars.p_ready[t], 128);
+            mbar_init(&bars.o_done[t], 1);
+        }
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(&bars.k_full[s], 1); mbar_init(&bars.k_empty[s], 1);
+            mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 0) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    volatile int* abortp = &abort_flag;
+
+    if (warp == 0 && lane == 0) {
+        // ------------------------------------------------------------ TMA producer
+        for (int t = 0; t < work.ntiles; ++t) {
+            mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
+            for (int s = 0; s < Cfg::SUB; ++s)
+                tma_load_2d(sQ + t * Cfg::TILE_BYTES + s * 16384, &maps.q, &bars.q_full[t], col0 + 64 * s,
+                            row0 + (work.tile0 + t) * TILE);
+        }
+        int jk = 0, jv = 0;
+        for (int j = 0; j < maxkv; ++j) {
+            if (!SYM) {
+                const int s = j % Cfg::KSTAGES;
+                if (j >= Cfg::KSTAGES && !mbar_wait(&bars.k_empty[s], ((j / Cfg::KSTAGES) - 1) & 1, abortp)) break;
+                mbar_arrive_expect_tx(&bars.k_full[s], Cfg::TILE_BYTES);
+                for (int u = 0; u < Cfg::SUB; ++u)
+                    tma_load_2d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], col0 + 64 * u,
+                                row0 + j * TILE);
+                jk = j + 1;
+            }
+            const int s = j % Cfg::VSTAGES;
+            if (j >= Cfg::VSTAGES && !mbar_wait(&bars.v_empty[s], ((j / Cfg::VSTAGES) - 1) & 1, abortp)) break;
+            mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
+            for (int u = 0; u < Cfg::SUB; ++u)
+                tma_load_2d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], col0 + 64 * u,
+                            row0 + j * TILE);
+            jv = j + 1;
+        }
+        if (*abortp) {  // let copies already issued land before shared memory is released
+            for (int t = 0; t < work.ntiles; ++t) mbar_wait_drain(&bars.q_full[t], 0);
+            for (int j = max(0, jk - Cfg::KSTAGES); j < jk; ++j)
+                mbar_wait_drain(&bars.k_full[j % Cfg::KSTAGES], (j / Cfg::KSTAGES) & 1);
+            for (int j = max(0, jv - Cfg::VSTAGES); j < jv; ++j)
+                mbar_wait_drain(&bars.v_full[j % Cfg::VSTAGES], (j / Cfg::VSTAGES) & 1);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ------------------------------------------------------------ MMA issuer
+        const uint32_t idescS = umma_idesc_bf16(128, 128, UMMA_K_MAJOR, UMMA_K_MAJOR);
+        const uint32_t idescO = umma_idesc_bf16(128, D, UMMA_K_MAJOR, UMMA_MN_MAJOR);
+        unsigned long long qk_blocks = 0, pv_blocks = 0;
+        bool ok = true;
+        auto issue_S = [&](int t, int j) -> bool {   // S_t = Q_t K_j^T        (phase 1, Eq. 1)
+            const int s = j % Cfg::KSTAGES;
+            if (!mbar_wait(&bars.k_full[s], (j / Cfg::KSTAGES) & 1, abortp)) return false;
+            tc_fence_after();
+            const uint32_t q = smem_u32(sQ + t * Cfg::TILE_BYTES), k = smem_u32(sK + s * Cfg::TILE_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
+                umma_ss(tmem + Cfg::TMEM_S + t * 128, umma_desc_kmajor(q + off), umma_desc_kmajor(k + off), idescS,
+                        kk != 0);
+            }
+            umma_commit(&bars.s_full[t]);
+            if (t == last_t) umma_commit(&bars.k_empty[s]);
+            ++qk_blocks;
+            return true;
+        };
+        auto issue_PV = [&](int t, int j) -> bool {  // O_t += P_t V_j         (phase 3, Eq. 3)
+            const int s = j % Cfg::VSTAGES;
+            if (!mbar_wait(&bars.p_ready[t], j & 1, abortp)) return false;
+            if (!mbar_wait(&bars.v_full[s], (j / Cfg::VSTAGES) & 1, abortp)) return false;
+            tc_fence_after();
+            const uint32_t v = smem_u32(sV + s * Cfg::TILE_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)
+                umma_ts(tmem + Cfg::TMEM_O + t * D, tmem + Cfg::TMEM_S + t * 128 + kk * 8,
+                        umma_desc_mnmajor(v + kk * 2048, 16384), idescO, (j | kk) != 0);
+            umma_commit(&bars.o_done[t]);
+            if (t == last_t) umma_commit(&bars.v_empty[s]);
+            ++pv_blocks;
+            return true;
+        };
+        for (int t = 0; t < work.ntiles && ok; ++t) ok = mbar_wait(&bars.q_full[t], 0, abortp);
+        if (!SYM)
+            for (int t = 0; t < work.ntiles && ok; ++t) ok = issue_S(t, 0);
+        for (int j = 0; j < maxkv && ok; ++j)
+            for (int t = 0; t < work.ntiles && ok; ++t)
+                if (j < nkv[t]) {
+                    ok = issue_PV(t, j);
+                    if (!SYM && ok && j + 1 < nkv[t]) ok = issue_S(t, j + 1);
+                }
+        const unsigned long long block_macs = (unsigned long long)TILE * TILE * D;
+        if (qk_blocks) atomicAdd(&dc->qk_macs, qk_blocks * block_macs);
+        if (pv_blocks) {
+            atomicAdd(&dc->pv_macs, pv_blocks * block_macs);
+            atomicAdd(&dc->exps, pv_blocks * (unsigned long long)(TILE * TILE));
+        }
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------ softmax + epilogue
+        const int t = (warp - 4) >> 2;
+        if (t < work.ntiles) {
+            const int q = warp & 3;
+            const int r = q * 32 + lane;                       // row inside the tile = TMEM lane
+            const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
+            const uint32_t tS = tmem + Cfg::TMEM_S + t * 128 + lane_off;
+            const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off;
+            const int It = work.tile0 + t;
+            const float* srow = SYM ? Sg + ((size_t)work.bh * n + (size_t)It * TILE + r) * n : nullptr;
+            float m_run = -INFINITY, l_run = 0.f;
+            bool ok = true;
+            for (int j = 0; j < nkv[t] && ok; ++j) {
+                if (!SYM) {
+                    ok = mbar_wait(&bars.s_full[t], j & 1, abortp);
+                } else if (j > 0) {
+                    ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);  // PV_{j-1} has consumed P
+                }
+                ok = __all_sync(0xffffffffu, ok);     // keep the warp together if one lane gave up
+                if (!ok) break;
+                tc_fence_after();
+                const bool diag = (scheme == PSA_MASKED) && (j == It);
+                // ---- pass 1: row maximum of the kept elements
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    if (!SYM) {
+                        tmem_ld32(tS + 32 * c, v);
+                        tc_wait_ld();
+                    } else {
+                        const float4* src = reinterpret_cast<const float4*>(srow + (size_t)j * TILE + 32 * c);
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const float4 f = __ldg(src + g);
+                            v[4 * g] = __float_as_uint(f.x); v[4 * g + 1] = __float_as_uint(f.y);
+                            v[4 * g + 2] = __float_as_uint(f.z); v[4 * g + 3] = __float_as_uint(f.w);
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float s = __uint_as_float(v[i]);
+                        if (!diag || (32 * c + i) <= r) mx = fmaxf(mx, s);
+                    }
+                }
+                const float mx2 = mx * sl2;
+                float alpha = 1.f;
+                if (mx2 > m_run + RESCALE_THRESHOLD) {   // also taken on the first tile (m_run = -inf)
+                    alpha = exp2f(m_run - mx2);
+                    m_run = mx2;
+                }
+                // ---- pass 2: P = exp2(S*sl2 - m), row sum, bf16 pack, store over S
+                float rowsum = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    if (!SYM) {
+                        tmem_ld32(tS + 32 * c, v);
+                        tc_wait_ld();
+                    } else {
+                        const float4* src = reinterpret_cast<const float4*>(srow + (size_t)j * TILE + 32 * c);
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const float4 f = __ldg(src + g);
+                            v[4 * g] = __float_as_uint(f.x); v[4 * g + 1] = __float_as_uint(f.y);
+                            v[4 * g + 2] = __float_as_uint(f.z); v[4 * g + 3] = __float_as_uint(f.w);
+                        }
+                    }
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float p0 = exp2f(fmaf(__uint_as_float(v[i]), sl2, -m_run));
+                        float p1 = exp2f(fmaf(__uint_as_float(v[i + 1]), sl2, -m_run));
+                        if (diag) {
+                            if (32 * c + i > r) p0 = 0.f;
+                            if (32 * c + i + 1 > r) p1 = 0.f;
+                        }
+                        rowsum += p0 + p1;
+                        pk[i >> 1] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st16(tS + 16 * c, pk);
+                }
+                l_run = l_run * alpha + rowsum;
+                // ---- rescale O when some row of this warp raised its maximum
+                if (j > 0) {
+                    if (!SYM) {
+                        ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);  // PV_{j-1} finished writing O
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
+                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t v[32];
+                            tmem_ld32(tO + 32 * c, v);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                            tmem_st32(tO + 32 * c, v);
+                        }
+                    }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(&bars.p_ready[t]);
+            }
+            if (ok) ok = mbar_wait(&bars.o_done[t], (nkv[t] - 1) & 1, abortp);
+            if (named_bar_all(ok, 2 + t, 128)) {
+                // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row)
+                tc_fence_after();
+                const float inv = 1.f / l_run;
+                uint8_t* stage = sQ + t * Cfg::TILE_BYTES;     // Q_t is no longer read by any MMA
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tO + c0, v);
+                    tc_wait_ld();
+                    uint8_t* sub = stage + (c0 / 64) * 16384;
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint4 o;
+                        o.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]) * inv, __uint_as_float(v[g * 8 + 1]) * inv);
+                        o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]) * inv, __uint_as_float(v[g * 8 + 3]) * inv);
+                        o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]) * inv, __uint_as_float(v[g * 8 + 5]) * inv);
+                        o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]) * inv, __uint_as_float(v[g * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4*>(sub + swz128_offset(r, (c0 % 64) / 8 + g)) = o;
+                    }
+                }
+                fence_async_smem();
+                named_bar_sync(2 + t, 128);
+                if (q == 0 && lane == 0) {
+                    for (int u = 0; u < Cfg::SUB; ++u)
+                        tma_store_2d(&maps.o, stage + u * 16384, col0 + 64 * u, row0 + It * TILE);
+                    tma_store_commit();
+                    tma_store_wait_all();
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicExch(&dc->status, (int)PSA_ERR_TIMEOUT);
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+// Phase 1 of the symmetric scheme (paper Sec. 4.1): one CTA per unordered tile pair {I, J}, J <= I,
+// computes S_IJ = scale * X_I X_J^T once and stores it at (I, J) and, transposed, at (J, I): the
+// mirror block costs stores, no MACs.  S: [heads_in_pass, n, n] fp32.
+template <int D>
+__global__ void __launch_bounds__(128, 2)
+sym_scores_kernel(const __grid_constant__ CUtensorMap mapX, float* __restrict__ Sg, int n, int H, int bh0,
+                  float scale, DeviceCounters* dc) {
+    constexpr int SUB = D / 64, TILE_BYTES = 128 * D * 2;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + TILE_BYTES;
+    __shared__ uint64_t full_bar, acc_bar;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_flag;
+    __shared__ float tr[4][32][33];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int T = row_tiles(n);
+    const int np = sym_pairs(T);
+    const int hl = blockIdx.x / np;                 // head inside this pass
+    int I, J;
+    sym_pair(blockIdx.x - hl * np, &I, &J);
+    const int bh = bh0 + hl, b = bh / H, h = bh - b * H;
+    const int row0 = b * n, col0 = h * D;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(&full_bar, 1);
+        mbar_init(&acc_bar, 1);
+        fence_mbar_init();
+    }
+    if (warp == 0) { tmem_alloc(&tmem_base_s, 128); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    volatile int* abortp = &abort_flag;
+
+    if (threadIdx.x == 0) {
+        mbar_arrive_expect_tx(&full_bar, 2 * TILE_BYTES);
+        for (int u = 0; u < SUB; ++u) {
+            tma_load_2d(sA + u * 16384, &mapX, &full_bar, col0 + 64 * u, row0 + I * TILE);
+            tma_load_2d(sB + u * 16384, &mapX, &full_bar, col0 + 64 * u, row0 + J * TILE);
+        }
+        if (mbar_wait(&full_bar, 0, abortp)) {
+            tc_fence_after();
+            const uint32_t idesc = umma_idesc_bf16(128, 128, UMMA_K_MAJOR, UMMA_K_MAJOR);
+            const uint32_t a = smem_u32(sA), bb = smem_u32(sB);
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
+                umma_ss(tmem, umma_desc_kmajor(a + off), umma_desc_kmajor(bb + off), idesc, kk != 0);
+            }
+            umma_commit(&acc_bar);
+            atomicAdd(&dc->qk_macs, (unsigned long long)TILE * TILE * D);
+        } else {
+            mbar_wait_drain(&full_bar, 0);
+        }
+    }
+    __syncwarp();
+    const bool ready = mbar_wait(&acc_bar, 0, abortp);
+    if (__syncthreads_and(ready)) {
+        tc_fence_after();
+        float* Sh = Sg + (size_t)hl * n * n;
+        const int r = warp * 32 + lane;
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem + (static_cast<uint32_t>(warp * 32) << 16) + c0, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float s = __uint_as_float(v[i]) * scale;
+                tr[warp][lane][i] = s;
+                if (I != J)  // mirror block: element (J*128 + c0 + i, I*128 + r); lanes run along a row
+                    Sh[((size_t)J * TILE + c0 + i) * n + (size_t)I * TILE + r] = s;
+            }
+            __syncwarp();
+#pragma unroll
+            for (int rr = 0; rr < 32; ++rr)  // direct block, lanes run along a row
+                Sh[((size_t)I * TILE + warp * 32 + rr) * n + (size_t)J * TILE + c0 + lane] = tr[warp][rr][lane];
+            __syncwarp();
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicExch(&dc->status, (int)PSA_ERR_TIMEOUT);
+    if (warp == 0) tmem_dealloc(tmem, 128);
+}
+
+constexpr size_t SYM_SCRATCH_CAP = size_t(2) << 30;  // bytes of score scratch per pass
+
+int sym_heads_per_pass(int B, int H, int n) {
+    const size_t per_head = (size_t)n * n * sizeof(float);
+    size_t hp = SYM_SCRATCH_CAP / per_head;
+    if (hp < 1) hp = 1;
+    if (hp > (size_t)B * H) hp = (size_t)B * H;
+    return (int)hp;
+}
+
+template <int D>
+int launch_attention(const void* Q, const void* K, const void* V, void* out, float* S, int B, int H, int n,
+                     float scale, int scheme, DeviceCounters* dc, cudaStream_t stream) {
+    using Cfg = AttnCfg<D>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(attn_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(sym_scores_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     2 * Cfg::TILE_BYTES + 1024);
+        if (e != cudaSuccess) { set_cuda_error(e, "cudaFuncSetAttribute(attention)"); return PSA_ERR_CUDA; }
+        attr_set = true;
+    }
+    const uint64_t rows = (uint64_t)B * n, cols = (uint64_t)H * D, pitch = cols * 2;
+    AttnMaps maps;
+    if (!make_tensor_map_bf16(&maps.q, Q, rows, cols, pitch, 128, 64) ||
+        !make_tensor_map_bf16(&maps.k, K, rows, cols, pitch, 128, 64) ||
+        !make_tensor_map_bf16(&maps.v, V, rows, cols, pitch, 128, 64) ||
+        !make_tensor_map_bf16(&maps.o, out, rows, cols, pitch, 128, 64))
+        return PSA_ERR_CUDA;
+    const int P = ctas_per_head(n);
+    cudaError_t e;
+    if (scheme != PSA_SYMMETRIC) {
+        attn_kernel<D, false><<<B * H * P, ATTN_THREADS, Cfg::SMEM, stream>>>(maps, nullptr, n, H, scheme, 0,
+                                                                             scale * LOG2E, dc);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { set_cuda_error(e, "attn_kernel launch"); return PSA_ERR_CUDA; }
+        return PSA_OK;
+    }
+    const int hp = sym_heads_per_pass(B, H, n);
+    const int np = sym_pairs(row_tiles(n));
+    for (int bh0 = 0; bh0 < B * H; bh0 += hp) {
+        const int heads = min(hp, B * H - bh0);
+        sym_scores_kernel<D><<<heads * np, 128, 2 * Cfg::TILE_BYTES + 1024, stream>>>(maps.q, S, n, H, bh0, scale, dc);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { set_cuda_error(e, "sym_scores_kernel launch"); return PSA_ERR_CUDA; }
+        attn_kernel<D, true><<<heads * P, ATTN_THREADS, Cfg::SMEM, stream>>>(maps, S, n, H, PSA_SYMMETRIC, bh0, LOG2E, dc);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { set_cuda_error(e, "attn_kernel(symmetric) launch"); return PSA_ERR_CUDA; }
+    }
+    return PSA_OK;
+}
+
+}  // namespace
+
+size_t bf16_symmetric_scratch_bytes(int B, int H, int n) {
+    return (size_t)sym_heads_per_pass(B, H, n) * n * n * sizeof(float);
+}
+
+int bf16_attention(const void* Q, const void* K, const void* V, void* out, float* S, size_t s_bytes, int B, int H,
+                   int n, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream) {
+    if (scheme == PSA_SYMMETRIC && (!S || s_bytes < bf16_symmetric_scratch_bytes(B, H, n))) return PSA_ERR_WORKSPACE;
+    if (d == 64) return launch_attention<64>(Q, K, V, out, S, B, H, n, scale, scheme, dc, stream);
+    if (d == 128) return launch_attention<128>(Q, K, V, out, S, B, H, n, scale, scheme, dc, stream);
+    return PSA_ERR_UNSUPPORTED;
+}
+
+}  // namespace psa

@@ -1,0 +1,201 @@
+// Projection GEMM for the bf16 path (paper Sec. 3.1: q, k, v = x*Wq, x*Wk, x*Wv):
+//     C_w[M, N] = A[M, K] * B_w[K, N],  w < nW,  bf16 row-major operands, fp32 accumulation in TMEM.
+//
+// One CTA per 128x128 output tile (two CTAs resident per SM so one tile's epilogue overlaps the
+// other's main loop).  Warp 0 streams operand tiles with TMA into a 3-stage shared-memory ring,
+// warp 1 issues tcgen05 MMAs (A K-major, B in its natural row-major form = MN-major), warps 2-5
+// move the accumulator TMEM -> registers -> bf16 -> swizzled shared memory -> TMA store.
+#include <stdio.h>
+
+#include <mutex>
+
+#include "psa_internal.h"
+#include "psa_tma.h"
+#include "sm100.cuh"
+
+namespace psa {
+
+// ---------------------------------------------------------------- tensor-map helper
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+std::once_flag g_encode_once;
+}  // namespace
+
+bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_bytes,
+                          uint32_t box_rows, uint32_t box_cols) {
+    std::call_once(g_encode_once, [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    });
+    if (!g_encode) { set_error_text("cuTensorMapEncodeTiled entry point not available"); return false; }
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {pitch_bytes};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t es[2] = {1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char msg[96];
+        snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        set_error_text(msg);
+        return false;
+    }
+    return true;
+}
+
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 64;
+constexpr int STAGES = 3;
+constexpr int A_BYTES = BM * BK * 2;           // 16 KB, K-major [128 x 64]
+constexpr int B_SUB_BYTES = BK * 64 * 2;       // 8 KB, one [64 k-rows x 64 n] sub-tile
+constexpr int B_BYTES = 2 * B_SUB_BYTES;       // 16 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES; // 32 KB
+constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024;  // + slack for 1024-byte alignment
+
+struct GemmMaps {
+    CUtensorMap a;
+    CUtensorMap b[3];
+    CUtensorMap c[3];
+};
+
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
+gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, DeviceCounters* dc) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_bar;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int w = blockIdx.z;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int nk = (K + BK - 1) / BK;
+    const CUtensorMap* mapB = &maps.b[w];
+    const CUtensorMap* mapC = &maps.c[w];
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&acc_bar, 1);
+        fence_mbar_init();
+    }
+    if (warp == 0) { tmem_alloc(&tmem_base_s, BN); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    volatile int* abortp = &abort_flag;
+
+    if (warp == 0 && lane == 0) {
+        // ---- TMA producer
+        int issued = 0;
+        for (int kt = 0; kt < nk; ++kt) {
+            const int s = kt % STAGES;
+            if (kt >= STAGES && !mbar_wait(&empty_bar[s], ((kt / STAGES) - 1) & 1, abortp)) break;
+            uint8_t* sA = smem + s * STAGE_BYTES;
+            uint8_t* sB = sA + A_BYTES;
+            mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
+            tma_load_2d(sA, &maps.a, &full_bar[s], kt * BK, m0);
+            tma_load_2d(sB, mapB, &full_bar[s], n0, kt * BK);
+            tma_load_2d(sB + B_SUB_BYTES, mapB, &full_bar[s], n0 + 64, kt * BK);
+            ++issued;
+        }
+        if (*abortp) {  // let copies already in flight land before the CTA goes away
+            for (int kt = max(0, issued - STAGES); kt < issued; ++kt)
+                mbar_wait_drain(&full_bar[kt % STAGES], (kt / STAGES) & 1);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---- MMA issuer
+        const uint32_t idesc = umma_idesc_bf16(BM, BN, UMMA_K_MAJOR, UMMA_MN_MAJOR);
+        bool ok = true;
+        for (int kt = 0; kt < nk && ok; ++kt) {
+            const int s = kt % STAGES;
+            ok = mbar_wait(&full_bar[s], (kt / STAGES) & 1, abortp);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t sA = smem_u32(smem + s * STAGE_BYTES), sB = sA + A_BYTES;
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k)
+                umma_ss(tmem, umma_desc_kmajor(sA + k * 32), umma_desc_mnmajor(sB + k * 2048, B_SUB_BYTES), idesc,
+                        (kt | k) != 0);
+            umma_commit(&empty_bar[s]);
+        }
+        if (ok) {
+            umma_commit(&acc_bar);
+            const unsigned long long vm = min(BM, M - m0), vn = min(BN, N - n0);
+            atomicAdd(&dc->proj_macs, vm * vn * (unsigned long long)K);
+        }
+    } else if (warp >= 2) {
+        // ---- epilogue: 4 warps, warp q owns TMEM lanes 32q .. 32q+31 = output rows
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const bool ready = mbar_wait(&acc_bar, 0, abortp);
+        if (named_bar_all(ready, 1, 128)) {  // uniform across the four epilogue warps
+            tc_fence_after();
+            uint8_t* stage = smem;  // the ring is drained: every load landed and every MMA completed
+#pragma unroll
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(tmem + (static_cast<uint32_t>(q * 32) << 16) + c0, r);
+                tc_wait_ld();
+                uint8_t* sub = stage + (c0 / 64) * (BM * 128);
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {  // four 16-byte chunks of 8 bf16
+                    uint4 v;
+                    v.x = pack_bf16x2(__uint_as_float(r[g * 8 + 0]), __uint_as_float(r[g * 8 + 1]));
+                    v.y = pack_bf16x2(__uint_as_float(r[g * 8 + 2]), __uint_as_float(r[g * 8 + 3]));
+                    v.z = pack_bf16x2(__uint_as_float(r[g * 8 + 4]), __uint_as_float(r[g * 8 + 5]));
+                    v.w = pack_bf16x2(__uint_as_float(r[g * 8 + 6]), __uint_as_float(r[g * 8 + 7]));
+                    *reinterpret_cast<uint4*>(sub + swz128_offset(row, (c0 % 64) / 8 + g)) = v;
+                }
+            }
+            fence_async_smem();
+            named_bar_sync(1, 128);
+            if (warp == 2 && lane == 0) {
+                tma_store_2d(mapC, stage, n0, m0);
+                if (n0 + 64 < N) tma_store_2d(mapC, stage + BM * 128, n0 + 64, m0);
+                tma_store_commit();
+                tma_store_wait_all();
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicExch(&dc->status, (int)PSA_ERR_TIMEOUT);
+    if (warp == 0) tmem_dealloc(tmem, BN);
+}
+
+}  // namespace
+
+int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int nW, int M, int K, int N,
+                 DeviceCounters* dc, cudaStream_t stream) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+        if (e != cudaSuccess) { set_cuda_error(e, "cudaFuncSetAttribute(gemm)"); return PSA_ERR_CUDA; }
+        attr_set = true;
+    }
+    GemmMaps maps;
+    if (!make_tensor_map_bf16(&maps.a, A, M, K, (uint64_t)K * 2, BM, BK)) return PSA_ERR_CUDA;
+    for (int w = 0; w < 3; ++w) {
+        const int src = w < nW ? w : 0;
+        if (!make_tensor_map_bf16(&maps.b[w], Bw[src], K, N, (uint64_t)N * 2, BK, 64)) return PSA_ERR_CUDA;
+        if (!make_tensor_map_bf16(&maps.c[w], C[src], M, N, (uint64_t)N * 2, BM, 64)) return PSA_ERR_CUDA;
+    }
+    dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM, nW);
+    gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(maps, M, N, K, dc);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error(e, "gemm_bf16_kernel launch"); return PSA_ERR_CUDA; }
+    return PSA_OK;
+}
+
+}  // namespace psa

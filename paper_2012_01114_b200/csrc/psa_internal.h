@@ -1,0 +1,41 @@
+// Internal declarations shared by the translation units of libpsa (not part of the public interface).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/psa.h"
+
+namespace psa {
+
+// Device-resident counters of one call, zeroed (stream-ordered) before its first kernel.
+// Kernels add to them once per block of work they actually issue.
+struct DeviceCounters {
+    unsigned long long proj_macs;
+    unsigned long long qk_macs;
+    unsigned long long pv_macs;
+    unsigned long long exps;
+    int status;  // PSA_OK or PSA_ERR_TIMEOUT
+    int pad;
+};
+
+// ---- fp32 CUDA-core path (psa_f32.cu) ----
+// out[w][r, c] = sum_k X[r, k] W[w][k, c] for w < nW.
+cudaError_t f32_project(const float* X, const float* const W[3], float* const out[3], int nW, int rows, int D,
+                        int N, DeviceCounters* dc, cudaStream_t stream);
+// Q, K, V, out: [B, n, H, d] fp32.  S: scratch [B*H, n, n] fp32, used by PSA_SYMMETRIC only.
+cudaError_t f32_attention(const float* Q, const float* K, const float* V, float* out, float* S, int B, int H,
+                          int n, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
+
+// ---- bf16 tcgen05 path (psa_gemm.cu, psa_attn.cu) ----
+// C[w][M, N] = A[M, K] * Bw[w][K, N], bf16 row-major, fp32 accumulation.  Returns a psa_status.
+int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int nW, int M, int K, int N,
+                 DeviceCounters* dc, cudaStream_t stream);
+// Q, K, V, out: [B, n, H, d] bf16.  S: scratch for PSA_SYMMETRIC ([heads_per_pass, n, n] fp32).
+int bf16_attention(const void* Q, const void* K, const void* V, void* out, float* S, size_t s_bytes, int B,
+                   int H, int n, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
+size_t bf16_symmetric_scratch_bytes(int B, int H, int n);
+
+void set_cuda_error(cudaError_t e, const char* where);
+void set_error_text(const char* text);
+
+}  // namespace psa

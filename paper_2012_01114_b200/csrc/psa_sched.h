@@ -1,0 +1,62 @@
+// Tile scheduler of the bf16 path: which 128x128 blocks of the weight matrix exist for a scheme,
+// and which CTA owns them.  Pure integer functions, compiled for both host and device so that the
+// analytic census (psa_skip_count) walks exactly the list the kernels walk.
+//
+// A block that the scheme makes redundant is absent from the list: it is never loaded, never
+// multiplied and never exponentiated (paper Sec. 4.1 for the symmetric scheme, Sec. 5.1 for the
+// masked one), as opposed to being computed and masked afterwards.
+#pragma once
+#include <stdint.h>
+
+#include "../../include/psa.h"
+
+#if defined(__CUDACC__)
+#define PSA_HD __host__ __device__ __forceinline__
+#else
+#define PSA_HD inline
+#endif
+
+namespace psa {
+
+constexpr int TILE = 128;          // rows and columns of one block of the weight matrix
+constexpr int TILES_PER_CTA = 2;   // a CTA owns two consecutive row tiles of one (batch, head)
+
+struct CtaWork {
+    int bh;        // batch * heads + head
+    int tile0;     // first row tile owned
+    int ntiles;    // 1 or 2 row tiles owned
+};
+
+PSA_HD int row_tiles(int n) { return n / TILE; }
+PSA_HD int ctas_per_head(int n) { return (row_tiles(n) + TILES_PER_CTA - 1) / TILES_PER_CTA; }
+
+// CTA index -> work.  Heads are the slow index so that CTAs resident together read the same K and
+// V (L2 reuse); inside a head the masked scheme hands out the heaviest row tiles first (the role of
+// the paper's pairing of long rows with short ones, Sec. 5.2: balance).
+PSA_HD CtaWork cta_work(int cta, int n, int scheme_masked) {
+    const int P = ctas_per_head(n);
+    CtaWork w;
+    w.bh = cta / P;
+    const int r = cta - w.bh * P;
+    const int p = scheme_masked ? (P - 1 - r) : r;
+    w.tile0 = p * TILES_PER_CTA;
+    const int left = row_tiles(n) - w.tile0;
+    w.ntiles = left < TILES_PER_CTA ? left : TILES_PER_CTA;
+    return w;
+}
+
+// Number of key/value tiles row tile I visits in phases 1-3 of the fused kernel (FULL, MASKED) or
+// in phases 2-3 (SYMMETRIC): column tiles 0 .. kv_tiles-1.
+PSA_HD int kv_tiles(int I, int T, int scheme) { return scheme == PSA_MASKED ? I + 1 : T; }
+
+// Phase 1 of the symmetric scheme: one block per unordered pair {I, J}; block t of a head,
+// t in [0, T(T+1)/2), is (I, J) with J <= I, enumerated row by row.
+PSA_HD void sym_pair(int t, int* I, int* J) {
+    int i = 0;
+    while ((i + 1) * (i + 2) / 2 <= t) ++i;
+    *I = i;
+    *J = t - i * (i + 1) / 2;
+}
+PSA_HD int sym_pairs(int T) { return T * (T + 1) / 2; }
+
+}  // namespace psa
