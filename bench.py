@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the self-attention hot path (projections -> scores -> softmax -> weighted sum).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl reference]
+
+One "step" is one pass of the whole path over one batch of a seeded synthetic workload
+(`paper_2012_01114_b200.inputs.WORKLOADS`).  The default workload is c3: batch 8, n = 1024,
+d_model = 768, 12 heads x 64, bf16, masked scheme, projections included.  Prints ONE JSON line.
+
+  value        useful TFLOP/s: 2 x (the paper's element-level MAC count for the scheme + the projection
+               MACs) / device time, inputs resident in HBM, CUDA events around each step
+  e2e          the same metric through psa_attention_host: host buffers in, host buffer out, copies timed
+  roofline     dominant kernel, timed by CUDA events recorded inside the library between its kernels
+  cpu_baseline the fp64 oracle timed on this machine's cores on a bounded sample of the same workload
+
+With N > 1 (torchrun) every rank runs its own replica of the workload on its own GPU: (batch, head)
+units are independent, there is no exchange step, so scaling is weak and the value is the sum over
+ranks divided by the slowest rank's time.  `--impl reference` times the oracle alone (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "useful attention TFLOP/s (non-skipped FLOPs)"
+UNIT = "TFLOP/s"
+L2_FLUSH_BYTES = 256 << 20
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def useful_flops(w, batch=None):
+    """2 x MACs the scheme needs at element level (paper Sec. 3.2, 4.2, 5.2) + projection MACs."""
+    B = w["batch"] if batch is None else batch
+    H, n, D, d = w["heads"], w["n"], w["d_model"], w["d_k"]
+    tri = n * (n + 1) // 2
+    qk = d * (n * n if w["scheme"] == 0 else tri)
+    pv = d * (tri if w["scheme"] == 2 else n * n)
+    proj = ((1 if w["scheme"] == 1 else 3) * n * D * H * d) if w["proj"] else 0
+    return {"core": 2.0 * B * H * (qk + pv), "proj": 2.0 * B * proj}
+
+
+def aggregate(per_rank_flops, max_seconds):
+    """Whole-job throughput in TFLOP/s from the sum of the ranks' work and the slowest rank's time."""
+    return float(sum(per_rank_flops)) / max_seconds / 1e12
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz, self._stop_evt = index, [], set(), None, threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or nv.nvmlDeviceGetCurrentClocksThrottleReasons
+                r = get(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_sample(w, seconds_budget=20.0):
+    """Times the oracle on a bounded sample of workload `w`: whole batch items (projection workloads) or
+    whole (batch, head) slices (core-only workloads).  Returns (TFLOP/s, cores, description)."""
+    import oracle
+    from paper_2012_01114_b200 import inputs
+    cores = os.cpu_count() or 1
+    name = w["name"]
+    if w["proj"]:
+        s = inputs.make(name)
+        v = s["values"]
+        done, t0 = 0, time.perf_counter()
+        while done < w["batch"]:       # whole batch items, until the budget is spent
+            oracle.attention_layer(v["X"][done:done + 1], v["Wq"], v.get("Wk", v["Wq"]), v.get("Wv", v["Wq"]),
+                                   w["heads"], w["scheme"])
+            done += 1
+            if time.perf_counter() - t0 > seconds_budget:
+                break
+        dt = time.perf_counter() - t0
+        fl = useful_flops(w, batch=done)
+        return (fl["core"] + fl["proj"]) / dt / 1e12, cores, "%d of %d batch items, all heads, projections included (%.1f s)" % (done, w["batch"], dt)
+    H, n, d = w["heads"], w["n"], w["d_k"]
+    sym = w["scheme"] == 1
+    q = inputs.tensor(w["seed"], 4, (1, n, H, d), 1.0, "bf16")[0]
+    k = q if sym else inputs.tensor(w["seed"], 5, (1, n, H, d), 1.0, "bf16")[0]
+    v = q if sym else inputs.tensor(w["seed"], 6, (1, n, H, d), 1.0, "bf16")[0]
+    per_slice = useful_flops(w, batch=1)["core"] / H
+    done, t0 = 0, time.perf_counter()
+    while done < H:
+        oracle.attention_core(q, k, v, w["scheme"], slices=[(0, done)])
+        done += 1
+        if time.perf_counter() - t0 > seconds_budget / 2:
+            break
+    dt = time.perf_counter() - t0
+    return per_slice * done / dt / 1e12, cores, "%d of %d (batch, head) slices in full (%.1f s)" % (done, w["batch"] * H, dt)
+
+
+def run_reference(args, w):
+    per_step = []
+    desc, cores = "", os.cpu_count() or 1
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        tf, cores, desc = oracle_sample(w, seconds_budget=12.0)
+        if i >= args.warmup:
+            per_step.append((tf, time.perf_counter() - t0))
+    val = float(np.mean([p[0] for p in per_step]))
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean([p[1] for p in per_step])),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_of(w, args), "gpu_launches": 0,
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def config_of(w, args):
+    from paper_2012_01114_b200 import inputs
+    return {"workload": w["name"], "batch": w["batch"], "heads": w["heads"], "n": w["n"], "d_model": w["d_model"] if w["proj"] else None,
+            "d_k": w["d_k"], "scheme": inputs.SCHEME_NAMES[w["scheme"]], "projections": bool(w["proj"]),
+            "parallelism": "replicas x%d (no exchange step)" % args.gpus,
+            "l2": "flushed between steps by an untimed %d MiB memset" % (L2_FLUSH_BYTES >> 20)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c3")
+    ap.add_argument("--impl", default="psa", choices=["psa", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer pass (for profiler captures)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "psa" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2012_01114_b200 import inputs
+    if args.impl == "reference":
+        if rank == 0:
+            w = dict(inputs.WORKLOADS[args.workload]); w["name"] = args.workload
+            run_reference(args, w)
+        return 0
+
+    import torch
+    import torch.distributed as dist
+    from paper_2012_01114_b200 import binding as psa, build
+    build.build()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    w = inputs.make(args.workload)
+    up = w["upload"]
+    H, scheme = w["heads"], w["scheme"]
+    sym = scheme == psa.SYMMETRIC
+
+    def bf16_host(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+
+    if w["proj"]:
+        host = {k: bf16_host(up[k]).pin_memory() for k in up}
+        dev = {k: t.cuda() for k, t in host.items()}
+        out = torch.empty((w["batch"], w["n"], H * w["d_k"]), dtype=torch.bfloat16, device="cuda")
+        out_host = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+
+        def step():
+            psa.psa_attention(dev["X"], dev["Wq"], dev.get("Wk"), dev.get("Wv"), H, scheme, out=out)
+        kernels_per_step = 2 + (1 if sym else 0)
+    else:
+        host = {k: bf16_host(up[k]).pin_memory() for k in up}
+        dev = {k: t.cuda() for k, t in host.items()}
+        out = torch.empty((w["batch"], w["n"], H * w["d_k"]), dtype=torch.bfloat16, device="cuda")
+        out_host = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+
+        def step():
+            psa.psa_attention_core(dev["Q"], dev.get("K"), dev.get("V"), scheme, out=out)
+        kernels_per_step = 1 + (1 if sym else 0)
+
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    fl = useful_flops(w)
+    flops_step = fl["core"] + fl["proj"]
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    torch.cuda.synchronize()
+    st, issued = psa.psa_last_issued()
+    if st != psa.OK:
+        raise RuntimeError("device status %d after warm-up" % st)
+
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    psa.psa_profile_begin(args.steps)
+    t_wall = time.perf_counter()
+    for s, e in ev:
+        flush.zero_()
+        s.record()
+        step()
+        e.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_wall = time.perf_counter() - t_wall
+    proj_ms, attn_ms, calls = psa.psa_profile_end()
+    clocks = sampler.stop()
+    step_ms = [s.elapsed_time(e) for s, e in ev]
+    total_s = sum(step_ms) / 1e3
+    if world > 1:
+        t = torch.tensor([total_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_s = float(t.item())
+    value = aggregate([flops_step * args.steps] * world, total_s)
+
+    # ---- end to end through the host-buffer entry point (copies inside the timed region)
+    e2e = None
+    if args.no_e2e:
+        n_e2e, e2e_s, h2d = 0, 1.0, 0
+    elif w["proj"]:
+        n_e2e = min(args.steps, 20)
+        for _ in range(2):
+            psa.psa_attention_host(host["X"], host["Wq"], host.get("Wk"), host.get("Wv"), H, scheme, out_host)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            psa.psa_attention_host(host["X"], host["Wq"], host.get("Wk"), host.get("Wv"), H, scheme, out_host)
+        e2e_s = time.perf_counter() - t0
+        h2d = sum(t.numel() * 2 for t in host.values())
+    else:
+        n_e2e = min(args.steps, 10)
+        e2e_stream = torch.cuda.current_stream()
+
+        def e2e_step():
+            for k in host:
+                dev[k].copy_(host[k], non_blocking=True)
+            step()
+            out_host.copy_(out, non_blocking=True)
+            e2e_stream.synchronize()
+        for _ in range(2):
+            e2e_step()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            e2e_step()
+        e2e_s = time.perf_counter() - t0
+        h2d = sum(t.numel() * 2 for t in host.values())
+    if world > 1:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = None if args.no_e2e else {"value": aggregate([flops_step * n_e2e] * world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": int(out_host.numel() * 2), "steps": n_e2e,
+           "api": "psa_attention_host" if w["proj"] else "pinned copies + psa_attention_core"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    peaks = measured_peaks()
+    issued_flops = {"proj": 2.0 * issued["proj_macs"], "core": 2.0 * (issued["qk_macs"] + issued["pv_macs"])}
+    kern = {"proj": proj_ms / max(calls, 1), "attn": attn_ms / max(calls, 1)}
+    dominant = "attn" if kern["attn"] >= kern["proj"] else "proj"
+    alg = fl["core"] if dominant == "attn" else fl["proj"]
+    achieved = alg / (kern[dominant] * 1e-3) / 1e12 if kern[dominant] > 0 else None
+    roofline = {"bound": "tensor", "kernel": "attn_kernel (fused scores-softmax-weighted sum)" if dominant == "attn" else "gemm_bf16_kernel (projections)",
+                "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": (achieved / peaks["bf16_tflops"]) if achieved else None, "peak_source": peaks["source"] + " burst bf16",
+                "traffic": None, "kernel_ms": kern, "algorithmic_flops": alg,
+                "issued_flops": issued_flops}
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        tf, cores, desc = oracle_sample(w)
+        cpu = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * total_s / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": config_of(w, args), "clocks": clocks, "e2e": e2e,
+            "gpu_launches": kernels_per_step * args.steps, "roofline": roofline, "cpu_baseline": cpu,
+            "pct_of_measured_bf16_peak": 100.0 * value / world / peaks["bf16_tflops"],
+            "pct_of_nominal_bf16_peak": 100.0 * value / world / 2250.0,
+            "skip": {"issued_macs": issued["qk_macs"] + issued["pv_macs"],
+                     "useful_macs": issued["useful_qk_macs"] + issued["useful_pv_macs"],
+                     "issued_fraction_of_full": (issued["qk_macs"] + issued["pv_macs"]) /
+                                                (2.0 * w["batch"] * H * w["d_k"] * w["n"] ** 2)},
+            "wall_s_timed_region": t_wall}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

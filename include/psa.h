@@ -130,6 +130,17 @@ size_t psa_workspace_bytes(int batch, int heads, int n, int d_model, int d_k, in
  */
 int psa_set_workspace(void* dev_ptr, size_t bytes);
 
+/*
+ * Per-kernel timing for benchmarks.  psa_profile_begin(max_calls) makes each of the next max_calls
+ * calls of psa_attention / psa_attention_f32 / psa_attention_core / psa_attention_host record CUDA
+ * events on the caller's stream before the projection kernel, between projection and attention,
+ * and after attention.  psa_profile_end waits for those events, returns the summed durations in
+ * milliseconds and the number of calls recorded, and releases the events.  Not thread-safe against
+ * concurrent attention calls.
+ */
+int psa_profile_begin(int max_calls);
+int psa_profile_end(float* proj_ms_sum, float* attn_ms_sum, int* calls);
+
 /* Text for a psa_status; never NULL. */
 const char* psa_status_string(int status);
 

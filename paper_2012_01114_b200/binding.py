@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "libpsa.so")
 
 EXPORTS = ("psa_attention", "psa_attention_f32", "psa_attention_core", "psa_attention_host", "psa_skip_count",
            "psa_last_issued", "psa_workspace_bytes", "psa_set_workspace", "psa_status_string",
-           "psa_last_cuda_error")
+           "psa_last_cuda_error", "psa_profile_begin", "psa_profile_end")
 
 
 class PsaError(RuntimeError):
@@ -66,6 +66,11 @@ def lib() -> ctypes.CDLL:
         L.psa_status_string.restype = ctypes.c_char_p
         L.psa_last_cuda_error.argtypes = []
         L.psa_last_cuda_error.restype = ctypes.c_char_p
+        L.psa_profile_begin.argtypes = [ci]
+        L.psa_profile_begin.restype = ci
+        L.psa_profile_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
+                                      ctypes.POINTER(ci)]
+        L.psa_profile_end.restype = ci
         for f in ("psa_attention", "psa_attention_f32", "psa_attention_core", "psa_attention_host",
                   "psa_skip_count", "psa_last_issued", "psa_set_workspace"):
             getattr(L, f).restype = ci
@@ -193,3 +198,18 @@ def psa_set_workspace(tensor):
     if rc != OK:
         raise PsaError(rc, "psa_set_workspace")
     _ws_keepalive = tensor
+
+
+def psa_profile_begin(max_calls: int):
+    rc = lib().psa_profile_begin(int(max_calls))
+    if rc != OK:
+        raise PsaError(rc, "psa_profile_begin")
+
+
+def psa_profile_end():
+    """(projection ms summed, attention ms summed, calls recorded) since psa_profile_begin."""
+    p, a, c = ctypes.c_float(), ctypes.c_float(), ctypes.c_int()
+    rc = lib().psa_profile_end(ctypes.byref(p), ctypes.byref(a), ctypes.byref(c))
+    if rc != OK:
+        raise PsaError(rc, "psa_profile_end")
+    return p.value, a.value, c.value

@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <mutex>
+#include <vector>
 
 #include "psa_internal.h"
 #include "psa_sched.h"
@@ -23,6 +24,8 @@ struct Context {
     size_t own_bytes = 0;
     int own_device = -1;
     DeviceCounters* last_dc = nullptr;  // counters of the most recent call
+    std::vector<cudaEvent_t> prof_events;  // 3 per profiled call
+    int prof_calls = 0, prof_max = 0;
     psa_counts last_useful = {0, 0, 0, 0, 0, 0};
 };
 Context g_ctx;
@@ -125,6 +128,13 @@ int run_layer(const void* X, const void* Wq, const void* Wk, const void* Wv, con
     useful_counts(batch, heads, n, d_model, d_k, scheme, with_proj, &g_ctx.last_useful);
     const float scale = 1.0f / sqrtf((float)d_k);
     const int nW = scheme == PSA_SYMMETRIC ? 1 : 3;
+    cudaEvent_t* pev = nullptr;
+    if (g_ctx.prof_calls < g_ctx.prof_max) pev = &g_ctx.prof_events[3 * g_ctx.prof_calls++];
+    struct EventTail {  // records the closing event on every exit path
+        cudaEvent_t* ev; cudaStream_t st;
+        ~EventTail() { if (ev) cudaEventRecord(ev[2], st); }
+    } tail{pev, stream};
+    if (pev) cudaEventRecord(pev[0], stream);
     if (with_proj) {
         void* outs[3] = {ws + L.q, ws + L.k, ws + L.v};
         const void* Ws[3] = {Wq, nW == 3 ? Wk : Wq, nW == 3 ? Wv : Wq};
@@ -138,6 +148,7 @@ int run_layer(const void* X, const void* Wq, const void* Wk, const void* Wv, con
         }
         Q = ws + L.q; K = ws + L.k; V = ws + L.v;
     }
+    if (pev) cudaEventRecord(pev[1], stream);
     float* S = scheme == PSA_SYMMETRIC ? reinterpret_cast<float*>(ws + L.s) : nullptr;
     if (dtype == PSA_F32) {
         e = f32_attention(static_cast<const float*>(Q), static_cast<const float*>(K), static_cast<const float*>(V),
@@ -320,6 +331,50 @@ int psa_set_workspace(void* dev_ptr, size_t bytes) {
     g_ctx.user_bytes = dev_ptr ? bytes : 0;
     g_ctx.last_dc = nullptr;
     return PSA_OK;
+}
+
+int psa_profile_begin(int max_calls) {
+    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    for (cudaEvent_t e : g_ctx.prof_events) cudaEventDestroy(e);
+    g_ctx.prof_events.clear();
+    g_ctx.prof_calls = 0;
+    g_ctx.prof_max = 0;
+    if (max_calls <= 0 || max_calls > 100000) return PSA_ERR_SHAPE;
+    g_ctx.prof_events.resize(3 * (size_t)max_calls);
+    for (size_t i = 0; i < g_ctx.prof_events.size(); ++i) {
+        cudaError_t e = cudaEventCreate(&g_ctx.prof_events[i]);
+        if (e != cudaSuccess) {
+            set_cuda_error(e, "cudaEventCreate");
+            for (size_t k = 0; k < i; ++k) cudaEventDestroy(g_ctx.prof_events[k]);
+            g_ctx.prof_events.clear();
+            return PSA_ERR_CUDA;
+        }
+    }
+    g_ctx.prof_max = max_calls;
+    return PSA_OK;
+}
+
+int psa_profile_end(float* proj_ms_sum, float* attn_ms_sum, int* calls) {
+    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    float p = 0.f, a = 0.f;
+    int rc = PSA_OK;
+    for (int c = 0; c < g_ctx.prof_calls; ++c) {
+        cudaEvent_t* ev = &g_ctx.prof_events[3 * c];
+        float t0 = 0.f, t1 = 0.f;
+        cudaError_t e = cudaEventSynchronize(ev[2]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&t0, ev[0], ev[1]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&t1, ev[1], ev[2]);
+        if (e != cudaSuccess) { set_cuda_error(e, "psa_profile_end"); rc = PSA_ERR_CUDA; break; }
+        p += t0; a += t1;
+    }
+    if (proj_ms_sum) *proj_ms_sum = p;
+    if (attn_ms_sum) *attn_ms_sum = a;
+    if (calls) *calls = g_ctx.prof_calls;
+    for (cudaEvent_t e : g_ctx.prof_events) cudaEventDestroy(e);
+    g_ctx.prof_events.clear();
+    g_ctx.prof_calls = 0;
+    g_ctx.prof_max = 0;
+    return rc;
 }
 
 const char* psa_status_string(int status) {
