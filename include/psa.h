@@ -141,6 +141,37 @@ int psa_set_workspace(void* dev_ptr, size_t bytes);
 int psa_profile_begin(int max_calls);
 int psa_profile_end(float* proj_ms_sum, float* attn_ms_sum, int* calls);
 
+/*
+ * Allocation-free variant of the fp32 symmetric-scheme attention core.  (The paper has no
+ * counterpart: this is a packaging of psa_attention_core(X, NULL, NULL, ..., PSA_SYMMETRIC, PSA_F32)
+ * for one kind of caller, not another algorithm.)
+ *
+ * Who it is for: callers that must not allocate device memory at call time -- a service whose device
+ * memory is budgeted and handed out once at start-up, a plug-in inside a host program that owns the
+ * allocator, a latency-critical loop where cudaMalloc (which may synchronise the whole device) is
+ * unacceptable.  The other entry points fall back on cudaMalloc for their workspace when none is
+ * registered; this one never calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ * How: the scratch the symmetric scheme needs (the score matrix S of every (batch, head), written once
+ * per unordered pair and mirrored, plus the operation counters) lives in a fixed array inside the
+ * library image, PSA_NOALLOC_SCRATCH_BYTES long.  Every GPU that loads the library holds that array
+ * until the process exits.
+ *
+ *   X     device, fp32, [batch, n, heads, d_k]: query = key = value        (caller-owned, read only)
+ *   out   device, fp32, [batch, n, heads*d_k]                              (caller-owned)
+ *   Limits: n <= 1024, d_k <= 128, and batch*heads*n*n <= PSA_NOALLOC_MAX_SCORES; a larger problem
+ *   returns PSA_ERR_WORKSPACE (psa_last_cuda_error() gives the sizes) and launches nothing.
+ *
+ * The first call on each device looks up the array's device address (with that device current); make
+ * that first call before starting any stream capture.  All calls share the one array, which keeps
+ * the previous call's contents: the call clears the counters it needs at zero and overwrites every
+ * score it later reads, but two calls whose kernels overlap on the GPU (different streams without an
+ * ordering between them) race on it -- order them.  psa_last_issued does not report on this entry.
+ */
+#define PSA_NOALLOC_MAX_SCORES (1u << 20)
+#define PSA_NOALLOC_SCRATCH_BYTES (256u + 4u * PSA_NOALLOC_MAX_SCORES)
+int psa_attention_sym_f32_noalloc(const void* X, int batch, int heads, int n, int d_k, void* out, void* stream);
+
 /* Text for a psa_status; never NULL. */
 const char* psa_status_string(int status);
 

@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "libpsa.so")
 
 EXPORTS = ("psa_attention", "psa_attention_f32", "psa_attention_core", "psa_attention_host", "psa_skip_count",
            "psa_last_issued", "psa_workspace_bytes", "psa_set_workspace", "psa_status_string",
-           "psa_last_cuda_error", "psa_profile_begin", "psa_profile_end")
+           "psa_last_cuda_error", "psa_profile_begin", "psa_profile_end", "psa_attention_sym_f32_noalloc")
 
 
 class PsaError(RuntimeError):
@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.psa_profile_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
                                       ctypes.POINTER(ci)]
         L.psa_profile_end.restype = ci
+        L.psa_attention_sym_f32_noalloc.argtypes = [vp, ci, ci, ci, ci, vp, vp]
+        L.psa_attention_sym_f32_noalloc.restype = ci
         for f in ("psa_attention", "psa_attention_f32", "psa_attention_core", "psa_attention_host",
                   "psa_skip_count", "psa_last_issued", "psa_set_workspace"):
             getattr(L, f).restype = ci
@@ -213,3 +215,23 @@ def psa_profile_end():
     if rc != OK:
         raise PsaError(rc, "psa_profile_end")
     return p.value, a.value, c.value
+
+
+def psa_attention_sym_f32_noalloc(X, out=None, stream=None):
+    """Symmetric-scheme fp32 attention core (query = key = value = X [B,n,H,d]) that allocates nothing:
+    its scratch is a fixed array inside the library, for callers that may not call cudaMalloc at run
+    time.  Problems with B*H*n*n above the built-in limit raise PsaError(ERR_WORKSPACE).  Pass `out`
+    to keep this wrapper allocation-free too."""
+    _check_dev(X, torch.float32, "X")
+    _check_dev(out, torch.float32, "out")
+    B, n, H, d = X.shape
+    if out is None:
+        out = torch.empty((B, n, H * d), dtype=torch.float32, device=X.device)
+    rc = lib().psa_attention_sym_f32_noalloc(_ptr(X), B, H, n, d, _ptr(out), _stream(stream))
+    if rc != OK:
+        detail = psa_last_cuda_error()
+        err = PsaError(rc, "psa_attention_sym_f32_noalloc")
+        if detail and rc == ERR_WORKSPACE:
+            err.args = (err.args[0] + ": " + detail,)
+        raise err
+    return out
