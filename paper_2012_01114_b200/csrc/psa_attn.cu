@@ -2,9 +2,9 @@
 // per pair of 128-row query tiles, never materialising the n x n weight matrix.
 //
 //   phase 1  S = Q K^T            tcgen05 MMA, operands staged by TMA, accumulator in TMEM
-//   phase 2  softmax              one thread per query row reads its row of S from TMEM, keeps a
+//   phase 2  softmax              two threads per query row (64 columns each) read S from TMEM, keep a
 //                                 running row maximum m and row sum l (the division of Eq. 2 is
-//                                 applied once to the output row), writes P = exp2(..) as bf16 back
+//                                 applied once to the output row), write P = exp2(..) as bf16 back
 //                                 into TMEM over S
 //   phase 3  O += P V             tcgen05 MMA with P read from TMEM and V (row-major = MN-major) from
 //                                 shared memory, accumulator O in TMEM
@@ -16,10 +16,20 @@
 // kernel that computes one block per unordered tile pair and stores it at both mirror positions;
 // this kernel then runs phases 2 and 3 reading S from that scratch.
 //
-// CTA layout (384 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 4-7 = softmax and
-// epilogue of row tile 0, warps 8-11 = the same for row tile 1.  The two row tiles ping-pong: while
-// the softmax warps of one work on S_j, the tensor core runs the other's MMAs.
-// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [256+D,256+2D); P_t overlays S_t.
+// CTA layout (576 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-9 = softmax and
+// epilogue of row tile 0, warps 10-17 = the same for row tile 1.  Within a tile's eight warps, warp
+// pairs (w, w+4) share a TMEM lane quarter (32 rows) and split the 128 columns of S in halves; the
+// pair agrees on the row maximum through shared memory.  The two row tiles ping-pong: while the
+// softmax warps of one work on S_j, the tensor core runs the other's MMAs.
+// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [256+D,256+2D); P_t (bf16, two per column)
+// overlays S_t: keys 0-63 at S_t columns [0,32), keys 64-127 at [64,96), each written by the thread that
+// owns that half of the row, so no thread overwrites scores another thread still has to read.
+//
+// exp2 is evaluated on the special-function unit for most elements and, for a fixed fraction of
+// them, by a degree-3 polynomial on the FMA pipe (range reduction by the round-to-nearest "magic
+// number" addition, exponent re-inserted with an integer add), because at these tile shapes the
+// special-function unit is as loaded as the tensor core.  Relative error of the polynomial:
+// 1.5e-4, well inside the bf16 rounding of P.
 #include "psa_internal.h"
 #include "psa_sched.h"
 #include "psa_tma.h"
@@ -29,7 +39,9 @@ namespace psa {
 
 namespace {
 
-constexpr int ATTN_THREADS = 384;
+constexpr int CTRL_WARPS = 2;                       // producer, MMA issuer
+constexpr int SOFTMAX_WARPS_PER_TILE = 8;
+constexpr int ATTN_THREADS = 32 * (CTRL_WARPS + 2 * SOFTMAX_WARPS_PER_TILE);   // 576
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float RESCALE_THRESHOLD = 8.0f;  // log2 units: O and l are rescaled only when the row max grew by more
 
@@ -41,6 +53,8 @@ struct AttnCfg {
     static constexpr int VSTAGES = D == 128 ? 2 : 4;
     static constexpr int SMEM = (2 + KSTAGES + VSTAGES) * TILE_BYTES + 1024;
     static constexpr int TMEM_S = 0, TMEM_O = 256;
+    // of every 4 consecutive elements, this many take the polynomial exp2 (FMA pipe) instead of MUFU
+    static constexpr int POLY_OF_4 = D == 128 ? 1 : 2;
 };
 
 struct AttnMaps {
@@ -52,6 +66,71 @@ struct AttnBars {
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
     uint64_t s_full[2], p_ready[2], o_done[2];
 };
+
+__device__ __forceinline__ float ex2_mufu(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// 2^x for x <= ~8 on the FMA pipe: n = round(x) by adding 1.5*2^23, f = x - n in [-0.5, 0.5],
+// 2^f by a cubic fitted to relative error 8e-5, then n is added into the exponent field.
+__device__ __forceinline__ float ex2_poly(float x) {
+    const float magic = 12582912.0f;
+    x = fmaxf(x, -126.0f);
+    const float t = __fadd_rn(x, magic);
+    const float f = __fsub_rn(x, __fsub_rn(t, magic));
+    float p = fmaf(f, 0.05508868396282196f, 0.24260404706001282f);
+    p = fmaf(p, f, 0.6932762265205383f);
+    p = fmaf(p, f, 0.9999289512634277f);
+    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// exp2 of 32 scores of one row (raw, unscaled) against the running maximum: P = exp2(s*sl2 - m), packed
+// to bf16 pairs in `pk`; returns the sum of the 32 weights (before rounding).  `col0` is the column of
+// s[0] inside the 128-wide block, used only by the diagonal predicate (j <= i kept).
+template <int POLY_OF_4, bool DIAG>
+__device__ __forceinline__ float exp_chunk32(const uint32_t (&s)[32], float sl2, float neg_m, int col0, int r,
+                                             uint32_t (&pk)[16]) {
+    float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        const float x0 = fmaf(__uint_as_float(s[i]), sl2, neg_m);
+        const float x1 = fmaf(__uint_as_float(s[i + 1]), sl2, neg_m);
+        float p0 = ((i & 3) < POLY_OF_4) ? ex2_poly(x0) : ex2_mufu(x0);
+        float p1 = (((i + 1) & 3) < POLY_OF_4) ? ex2_poly(x1) : ex2_mufu(x1);
+        if (DIAG) {
+            if (col0 + i > r) p0 = 0.f;
+            if (col0 + i + 1 > r) p1 = 0.f;
+        }
+        sum0 += p0;
+        sum1 += p1;
+        pk[i >> 1] = pack_bf16x2(p0, p1);
+    }
+    return sum0 + sum1;
+}
+
+template <bool DIAG>
+__device__ __forceinline__ float max_chunk32(const uint32_t (&s)[32], int col0, int r, float mx) {
+    if (!DIAG) {
+        float a = mx, b = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            a = max3(a, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+            b = max3(b, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        }
+        return fmaxf(a, b);
+    }
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        if (col0 + i <= r) mx = fmaxf(mx, __uint_as_float(s[i]));
+    return mx;
+}
+
 
 template <int D, bool SYM>
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
@@ -66,6 +145,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
     __shared__ AttnBars bars;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
+    __shared__ float xch_max[2][2][2][128];   // [step parity][tile][column half][row]
+    __shared__ float xch_sum[2][2][128];      // [tile][column half][row]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int T = row_tiles(n);
@@ -73,10 +154,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
     const int bh = bh0 + work.bh;
     const int b = bh / H, h = bh - b * H;
     const int row0 = b * n, col0 = h * D;
-    int nkv[2];
-    nkv[0] = kv_tiles(work.tile0, T, scheme);
-    nkv[1] = work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0;
-    const int maxkv = max(nkv[0], nkv[1]);
+    const int nkv0 = kv_tiles(work.tile0, T, scheme);
+    const int nkv1 = work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0;
+    const int maxkv = max(nkv0, nkv1);
     const int last_t = work.ntiles - 1;
 
     if (threadIdx.x == 0) {
@@ -84,7 +164,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bars.q_full[t], 1);
             mbar_init(&bars.s_full[t], 1);
-            mbar_init(&bars.p_ready[t], 128);
+            mbar_init(&bars.p_ready[t], 32 * SOFTMAX_WARPS_PER_TILE);
             mbar_init(&bars.o_done[t], 1);
         }
         for (int s = 0; s < 4; ++s) {
@@ -100,123 +180,125 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
     const uint32_t tmem = tmem_base_s;
     volatile int* abortp = &abort_flag;
 
-    if (warp == 0 && lane == 0) {
-        // ------------------------------------------------------------ TMA producer
-        for (int t = 0; t < work.ntiles; ++t) {
-            mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
-            for (int s = 0; s < Cfg::SUB; ++s)
-                tma_load_2d(sQ + t * Cfg::TILE_BYTES + s * 16384, &maps.q, &bars.q_full[t], col0 + 64 * s,
-                            row0 + (work.tile0 + t) * TILE);
-        }
-        int jk = 0, jv = 0;
-        for (int j = 0; j < maxkv; ++j) {
-            if (!SYM) {
-                const int s = j % Cfg::KSTAGES;
-                if (j >= Cfg::KSTAGES && !mbar_wait(&bars.k_empty[s], ((j / Cfg::KSTAGES) - 1) & 1, abortp)) break;
-                mbar_arrive_expect_tx(&bars.k_full[s], Cfg::TILE_BYTES);
-                for (int u = 0; u < Cfg::SUB; ++u)
-                    tma_load_2d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], col0 + 64 * u,
-                                row0 + j * TILE);
-                jk = j + 1;
+    if (warp == 0) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ TMA producer
+            for (int t = 0; t < work.ntiles; ++t) {
+                mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
+                for (int s = 0; s < Cfg::SUB; ++s)
+                    tma_load_2d(sQ + t * Cfg::TILE_BYTES + s * 16384, &maps.q, &bars.q_full[t], col0 + 64 * s,
+                                row0 + (work.tile0 + t) * TILE);
             }
-            const int s = j % Cfg::VSTAGES;
-            if (j >= Cfg::VSTAGES && !mbar_wait(&bars.v_empty[s], ((j / Cfg::VSTAGES) - 1) & 1, abortp)) break;
-            mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
-            for (int u = 0; u < Cfg::SUB; ++u)
-                tma_load_2d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], col0 + 64 * u,
-                            row0 + j * TILE);
-            jv = j + 1;
-        }
-        if (*abortp) {  // let copies already issued land before shared memory is released
-            for (int t = 0; t < work.ntiles; ++t) mbar_wait_drain(&bars.q_full[t], 0);
-            for (int j = max(0, jk - Cfg::KSTAGES); j < jk; ++j)
-                mbar_wait_drain(&bars.k_full[j % Cfg::KSTAGES], (j / Cfg::KSTAGES) & 1);
-            for (int j = max(0, jv - Cfg::VSTAGES); j < jv; ++j)
-                mbar_wait_drain(&bars.v_full[j % Cfg::VSTAGES], (j / Cfg::VSTAGES) & 1);
-        }
-    } else if (warp == 1 && lane == 0) {
-        // ------------------------------------------------------------ MMA issuer
-        const uint32_t idescS = umma_idesc_bf16(128, 128, UMMA_K_MAJOR, UMMA_K_MAJOR);
-        const uint32_t idescO = umma_idesc_bf16(128, D, UMMA_K_MAJOR, UMMA_MN_MAJOR);
-        unsigned long long qk_blocks = 0, pv_blocks = 0;
-        bool ok = true;
-        auto issue_S = [&](int t, int j) -> bool {   // S_t = Q_t K_j^T        (phase 1, Eq. 1)
-            const int s = j % Cfg::KSTAGES;
-            if (!mbar_wait(&bars.k_full[s], (j / Cfg::KSTAGES) & 1, abortp)) return false;
-            tc_fence_after();
-            const uint32_t q = smem_u32(sQ + t * Cfg::TILE_BYTES), k = smem_u32(sK + s * Cfg::TILE_BYTES);
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
-                umma_ss(tmem + Cfg::TMEM_S + t * 128, umma_desc_kmajor(q + off), umma_desc_kmajor(k + off), idescS,
-                        kk != 0);
-            }
-            umma_commit(&bars.s_full[t]);
-            if (t == last_t) umma_commit(&bars.k_empty[s]);
-            ++qk_blocks;
-            return true;
-        };
-        auto issue_PV = [&](int t, int j) -> bool {  // O_t += P_t V_j         (phase 3, Eq. 3)
-            const int s = j % Cfg::VSTAGES;
-            if (!mbar_wait(&bars.p_ready[t], j & 1, abortp)) return false;
-            if (!mbar_wait(&bars.v_full[s], (j / Cfg::VSTAGES) & 1, abortp)) return false;
-            tc_fence_after();
-            const uint32_t v = smem_u32(sV + s * Cfg::TILE_BYTES);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                umma_ts(tmem + Cfg::TMEM_O + t * D, tmem + Cfg::TMEM_S + t * 128 + kk * 8,
-                        umma_desc_mnmajor(v + kk * 2048, 16384), idescO, (j | kk) != 0);
-            umma_commit(&bars.o_done[t]);
-            if (t == last_t) umma_commit(&bars.v_empty[s]);
-            ++pv_blocks;
-            return true;
-        };
-        for (int t = 0; t < work.ntiles && ok; ++t) ok = mbar_wait(&bars.q_full[t], 0, abortp);
-        if (!SYM)
-            for (int t = 0; t < work.ntiles && ok; ++t) ok = issue_S(t, 0);
-        for (int j = 0; j < maxkv && ok; ++j)
-            for (int t = 0; t < work.ntiles && ok; ++t)
-                if (j < nkv[t]) {
-                    ok = issue_PV(t, j);
-                    if (!SYM && ok && j + 1 < nkv[t]) ok = issue_S(t, j + 1);
+            int jk = 0, jv = 0;
+            for (int j = 0; j < maxkv; ++j) {
+                if (!SYM) {
+                    const int s = j % Cfg::KSTAGES;
+                    if (j >= Cfg::KSTAGES && !mbar_wait(&bars.k_empty[s], ((j / Cfg::KSTAGES) - 1) & 1, abortp)) break;
+                    mbar_arrive_expect_tx(&bars.k_full[s], Cfg::TILE_BYTES);
+                    for (int u = 0; u < Cfg::SUB; ++u)
+                        tma_load_2d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], col0 + 64 * u,
+                                    row0 + j * TILE);
+                    jk = j + 1;
                 }
-        const unsigned long long block_macs = (unsigned long long)TILE * TILE * D;
-        if (qk_blocks) atomicAdd(&dc->qk_macs, qk_blocks * block_macs);
-        if (pv_blocks) {
-            atomicAdd(&dc->pv_macs, pv_blocks * block_macs);
-            atomicAdd(&dc->exps, pv_blocks * (unsigned long long)(TILE * TILE));
+                const int s = j % Cfg::VSTAGES;
+                if (j >= Cfg::VSTAGES && !mbar_wait(&bars.v_empty[s], ((j / Cfg::VSTAGES) - 1) & 1, abortp)) break;
+                mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
+                for (int u = 0; u < Cfg::SUB; ++u)
+                    tma_load_2d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], col0 + 64 * u,
+                                row0 + j * TILE);
+                jv = j + 1;
+            }
+            if (*abortp) {  // let copies already issued land before shared memory is released
+                for (int t = 0; t < work.ntiles; ++t) mbar_wait_drain(&bars.q_full[t], 0);
+                for (int j = max(0, jk - Cfg::KSTAGES); j < jk; ++j)
+                    mbar_wait_drain(&bars.k_full[j % Cfg::KSTAGES], (j / Cfg::KSTAGES) & 1);
+                for (int j = max(0, jv - Cfg::VSTAGES); j < jv; ++j)
+                    mbar_wait_drain(&bars.v_full[j % Cfg::VSTAGES], (j / Cfg::VSTAGES) & 1);
+            }
         }
-    } else if (warp >= 4) {
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ MMA issuer
+            const uint32_t idescS = umma_idesc_bf16(128, 128, UMMA_K_MAJOR, UMMA_K_MAJOR);
+            const uint32_t idescO = umma_idesc_bf16(128, D, UMMA_K_MAJOR, UMMA_MN_MAJOR);
+            unsigned long long qk_blocks = 0, pv_blocks = 0;
+            bool ok = true;
+            auto issue_S = [&](int t, int j) -> bool {   // S_t = Q_t K_j^T        (phase 1, Eq. 1)
+                const int s = j % Cfg::KSTAGES;
+                if (!mbar_wait(&bars.k_full[s], (j / Cfg::KSTAGES) & 1, abortp)) return false;
+                tc_fence_after();
+                const uint32_t q = smem_u32(sQ + t * Cfg::TILE_BYTES), k = smem_u32(sK + s * Cfg::TILE_BYTES);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
+                    umma_ss(tmem + Cfg::TMEM_S + t * 128, umma_desc_kmajor(q + off), umma_desc_kmajor(k + off), idescS,
+                            kk != 0);
+                }
+                umma_commit(&bars.s_full[t]);
+                if (t == last_t) umma_commit(&bars.k_empty[s]);
+                ++qk_blocks;
+                return true;
+            };
+            auto issue_PV = [&](int t, int j) -> bool {  // O_t += P_t V_j         (phase 3, Eq. 3)
+                const int s = j % Cfg::VSTAGES;
+                if (!mbar_wait(&bars.p_ready[t], j & 1, abortp)) return false;
+                if (!mbar_wait(&bars.v_full[s], (j / Cfg::VSTAGES) & 1, abortp)) return false;
+                tc_fence_after();
+                const uint32_t v = smem_u32(sV + s * Cfg::TILE_BYTES);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    umma_ts(tmem + Cfg::TMEM_O + t * D, tmem + Cfg::TMEM_S + t * 128 + (kk >> 2) * 64 + (kk & 3) * 8,
+                            umma_desc_mnmajor(v + kk * 2048, 16384), idescO, (j | kk) != 0);
+                umma_commit(&bars.o_done[t]);
+                if (t == last_t) umma_commit(&bars.v_empty[s]);
+                ++pv_blocks;
+                return true;
+            };
+            for (int t = 0; t < work.ntiles && ok; ++t) ok = mbar_wait(&bars.q_full[t], 0, abortp);
+            if (!SYM)
+                for (int t = 0; t < work.ntiles && ok; ++t) ok = issue_S(t, 0);
+            for (int j = 0; j < maxkv && ok; ++j)
+                for (int t = 0; t < work.ntiles && ok; ++t)
+                    if (j < (t == 0 ? nkv0 : nkv1)) {
+                        ok = issue_PV(t, j);
+                        if (!SYM && ok && j + 1 < (t == 0 ? nkv0 : nkv1)) ok = issue_S(t, j + 1);
+                    }
+            const unsigned long long block_macs = (unsigned long long)TILE * TILE * D;
+            if (qk_blocks) atomicAdd(&dc->qk_macs, qk_blocks * block_macs);
+            if (pv_blocks) {
+                atomicAdd(&dc->pv_macs, pv_blocks * block_macs);
+                atomicAdd(&dc->exps, pv_blocks * (unsigned long long)(TILE * TILE));
+            }
+        }
+    } else {
         // ------------------------------------------------------------ softmax + epilogue
-        const int t = (warp - 4) >> 2;
+        const int sw = warp - CTRL_WARPS;
+        const int t = sw >> 3;                                  // row tile of this warp
+        const int hlf = (sw >> 2) & 1;                          // column half of S / O this thread owns
+        const int nkv = t == 0 ? nkv0 : nkv1;
         if (t < work.ntiles) {
-            const int q = warp & 3;
-            const int r = q * 32 + lane;                       // row inside the tile = TMEM lane
+            const int q = warp & 3;                             // TMEM lane quarter this warp may access
+            const int r = q * 32 + lane;                        // row inside the tile = TMEM lane
             const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
             const uint32_t tS = tmem + Cfg::TMEM_S + t * 128 + lane_off;
-            const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off;
+            const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off + hlf * (D / 2);
             const int It = work.tile0 + t;
-            const float* srow = SYM ? Sg + ((size_t)work.bh * n + (size_t)It * TILE + r) * n : nullptr;
+            const int pair_bar = 1 + t * 4 + q;                 // named barrier of the two warps sharing rows
+            const int tile_bar = 9 + t;                         // named barrier of the tile's eight warps
+            const int col_base = hlf * 64;
+            const float* srow = SYM ? Sg + ((size_t)work.bh * n + (size_t)It * TILE + r) * n + col_base : nullptr;
             float m_run = -INFINITY, l_run = 0.f;
             bool ok = true;
-            for (int j = 0; j < nkv[t] && ok; ++j) {
-                if (!SYM) {
-                    ok = mbar_wait(&bars.s_full[t], j & 1, abortp);
-                } else if (j > 0) {
-                    ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);  // PV_{j-1} has consumed P
-                }
-                ok = __all_sync(0xffffffffu, ok);     // keep the warp together if one lane gave up
-                if (!ok) break;
-                tc_fence_after();
+            for (int j = 0; j < nkv; ++j) {
+                if (!SYM) ok = mbar_wait(&bars.s_full[t], j & 1, abortp);
+                if (ok && j > 0) ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);  // PV_{j-1} done with P and O
+                ok = __all_sync(0xffffffffu, ok);
                 const bool diag = (scheme == PSA_MASKED) && (j == It);
-                // ---- pass 1: row maximum of the kept elements
                 float mx = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
+                // 32 raw scores of this thread's half row: chunk c covers block columns col_base + 32c ..
+                auto load32 = [&](int c, uint32_t (&v)[32]) {
                     if (!SYM) {
-                        tmem_ld32(tS + 32 * c, v);
-                        tc_wait_ld();
+                        tmem_ld32(tS + col_base + 32 * c, v);
                     } else {
                         const float4* src = reinterpret_cast<const float4*>(srow + (size_t)j * TILE + 32 * c);
 #pragma unroll
@@ -226,86 +308,76 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                             v[4 * g + 2] = __float_as_uint(f.z); v[4 * g + 3] = __float_as_uint(f.w);
                         }
                     }
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float s = __uint_as_float(v[i]);
-                        if (!diag || (32 * c + i) <= r) mx = fmaxf(mx, s);
+                };
+                if (ok) {
+                    // ---- pass 1: maximum of this thread's 64 scores
+                    tc_fence_after();
+                    uint32_t a[32], bb[32];
+                    load32(0, a);
+                    load32(1, bb);
+                    if (!SYM) tc_wait_ld();
+                    if (diag) {
+                        mx = max_chunk32<true>(a, col_base, r, mx);
+                        mx = max_chunk32<true>(bb, col_base + 32, r, mx);
+                    } else {
+                        mx = max_chunk32<false>(a, col_base, r, mx);
+                        mx = max_chunk32<false>(bb, col_base + 32, r, mx);
                     }
+                    xch_max[j & 1][t][hlf][r] = mx;
                 }
+                // The two threads of a row meet here to exchange their half-row maxima (and to leave
+                // together if either gave up a wait).
+                ok = named_bar_all(ok, pair_bar, 64);
+                if (!ok) break;
+                mx = fmaxf(mx, xch_max[j & 1][t][hlf ^ 1][r]);
                 const float mx2 = mx * sl2;
                 float alpha = 1.f;
-                if (mx2 > m_run + RESCALE_THRESHOLD) {   // also taken on the first tile (m_run = -inf)
-                    alpha = exp2f(m_run - mx2);
+                if (mx2 > m_run + RESCALE_THRESHOLD) {   // also taken on the first block (m_run = -inf)
+                    alpha = ex2_mufu(m_run - mx2);
                     m_run = mx2;
                 }
-                // ---- pass 2: P = exp2(S*sl2 - m), row sum, bf16 pack, store over S
+                // ---- pass 2: P = exp2(S*sl2 - m) as bf16, stored over this thread's own half of S
+                // (columns [col_base, col_base + 32) of the block's TMEM region), behind its own reads.
                 float rowsum = 0.f;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    if (!SYM) {
-                        tmem_ld32(tS + 32 * c, v);
-                        tc_wait_ld();
-                    } else {
-                        const float4* src = reinterpret_cast<const float4*>(srow + (size_t)j * TILE + 32 * c);
-#pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            const float4 f = __ldg(src + g);
-                            v[4 * g] = __float_as_uint(f.x); v[4 * g + 1] = __float_as_uint(f.y);
-                            v[4 * g + 2] = __float_as_uint(f.z); v[4 * g + 3] = __float_as_uint(f.w);
-                        }
-                    }
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float p0 = exp2f(fmaf(__uint_as_float(v[i]), sl2, -m_run));
-                        float p1 = exp2f(fmaf(__uint_as_float(v[i + 1]), sl2, -m_run));
-                        if (diag) {
-                            if (32 * c + i > r) p0 = 0.f;
-                            if (32 * c + i + 1 > r) p1 = 0.f;
-                        }
-                        rowsum += p0 + p1;
-                        pk[i >> 1] = pack_bf16x2(p0, p1);
-                    }
-                    tmem_st16(tS + 16 * c, pk);
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t v[32], pk[16];
+                    load32(c, v);
+                    if (!SYM) tc_wait_ld();
+                    rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(v, sl2, -m_run, col_base + 32 * c, r, pk)
+                                   : exp_chunk32<Cfg::POLY_OF_4, false>(v, sl2, -m_run, col_base + 32 * c, r, pk);
+                    tmem_st16(tS + col_base + 16 * c, pk);
                 }
-                l_run = l_run * alpha + rowsum;
-                // ---- rescale O when some row of this warp raised its maximum
-                if (j > 0) {
-                    if (!SYM) {
-                        ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);  // PV_{j-1} finished writing O
-                        ok = __all_sync(0xffffffffu, ok);
-                        if (!ok) break;
-                        tc_fence_after();
-                    }
-                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                l_run = fmaf(l_run, alpha, rowsum);
+                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8
 #pragma unroll
-                        for (int c = 0; c < D / 32; ++c) {
-                            uint32_t v[32];
-                            tmem_ld32(tO + 32 * c, v);
-                            tc_wait_ld();
+                    for (int c = 0; c < D / 64; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tO + 32 * c, v);
+                        tc_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                            tmem_st32(tO + 32 * c, v);
-                        }
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                        tmem_st32(tO + 32 * c, v);
                     }
                 }
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(&bars.p_ready[t]);
             }
-            if (ok) ok = mbar_wait(&bars.o_done[t], (nkv[t] - 1) & 1, abortp);
-            if (named_bar_all(ok, 2 + t, 128)) {
+            if (ok) ok = mbar_wait(&bars.o_done[t], (nkv - 1) & 1, abortp);
+            xch_sum[t][hlf][r] = l_run;
+            if (named_bar_all(ok, tile_bar, 32 * SOFTMAX_WARPS_PER_TILE)) {
                 // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row)
                 tc_fence_after();
-                const float inv = 1.f / l_run;
+                const float inv = 1.f / (l_run + xch_sum[t][hlf ^ 1][r]);
                 uint8_t* stage = sQ + t * Cfg::TILE_BYTES;     // Q_t is no longer read by any MMA
 #pragma unroll
-                for (int c0 = 0; c0 < D; c0 += 32) {
+                for (int c = 0; c < D / 64; ++c) {
+                    const int col = hlf * (D / 2) + 32 * c;    // first of 32 output columns handled here
                     uint32_t v[32];
-                    tmem_ld32(tO + c0, v);
+                    tmem_ld32(tO + 32 * c, v);
                     tc_wait_ld();
-                    uint8_t* sub = stage + (c0 / 64) * 16384;
+                    uint8_t* sub = stage + (col / 64) * 16384;
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         uint4 o;
@@ -313,12 +385,12 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                         o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]) * inv, __uint_as_float(v[g * 8 + 3]) * inv);
                         o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]) * inv, __uint_as_float(v[g * 8 + 5]) * inv);
                         o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]) * inv, __uint_as_float(v[g * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(sub + swz128_offset(r, (c0 % 64) / 8 + g)) = o;
+                        *reinterpret_cast<uint4*>(sub + swz128_offset(r, (col % 64) / 8 + g)) = o;
                     }
                 }
                 fence_async_smem();
-                named_bar_sync(2 + t, 128);
-                if (q == 0 && lane == 0) {
+                named_bar_sync(tile_bar, 32 * SOFTMAX_WARPS_PER_TILE);
+                if (sw == t * 8 && lane == 0) {
                     for (int u = 0; u < Cfg::SUB; ++u)
                         tma_store_2d(&maps.o, stage + u * 16384, col0 + 64 * u, row0 + It * TILE);
                     tma_store_commit();
@@ -332,6 +404,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
     if (threadIdx.x == 0 && abort_flag) atomicExch(&dc->status, (int)PSA_ERR_TIMEOUT);
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
+
 
 // Phase 1 of the symmetric scheme (paper Sec. 4.1): one CTA per unordered tile pair {I, J}, J <= I,
 // computes S_IJ = scale * X_I X_J^T once and stores it at (I, J) and, transposed, at (J, I): the
