@@ -39,6 +39,9 @@ namespace psa {
 
 namespace {
 
+#ifndef PSA_POLY_OF_4
+#define PSA_POLY_OF_4 0
+#endif
 constexpr int CTRL_WARPS = 2;                       // producer, MMA issuer
 constexpr int SOFTMAX_WARPS_PER_TILE = 8;
 constexpr int ATTN_THREADS = 32 * (CTRL_WARPS + 2 * SOFTMAX_WARPS_PER_TILE);   // 576
@@ -54,7 +57,7 @@ struct AttnCfg {
     static constexpr int SMEM = (2 + KSTAGES + VSTAGES) * TILE_BYTES + 1024;
     static constexpr int TMEM_S = 0, TMEM_O = 256;
     // of every 4 consecutive elements, this many take the polynomial exp2 (FMA pipe) instead of MUFU
-    static constexpr int POLY_OF_4 = D == 128 ? 1 : 2;
+    static constexpr int POLY_OF_4 = PSA_POLY_OF_4;
 };
 
 struct AttnMaps {
@@ -223,16 +226,22 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
             const uint32_t idescO = umma_idesc_bf16(128, D, UMMA_K_MAJOR, UMMA_MN_MAJOR);
             unsigned long long qk_blocks = 0, pv_blocks = 0;
             bool ok = true;
+            // Descriptor low words of the operand bases; per MMA only a constant is added (sm100.cuh).
+            const uint32_t q_lo0 = umma_desc_lo_kmajor(smem_u32(sQ)), q_lo1 = umma_desc_lo_kmajor(smem_u32(sQ + Cfg::TILE_BYTES));
+            const uint32_t k_lo = umma_desc_lo_kmajor(smem_u32(sK));
+            const uint32_t v_lo = umma_desc_lo_mnmajor(smem_u32(sV), 16384);
+            const uint32_t tS0 = tmem + Cfg::TMEM_S, tO0 = tmem + Cfg::TMEM_O;
             auto issue_S = [&](int t, int j) -> bool {   // S_t = Q_t K_j^T        (phase 1, Eq. 1)
                 const int s = j % Cfg::KSTAGES;
                 if (!mbar_wait(&bars.k_full[s], (j / Cfg::KSTAGES) & 1, abortp)) return false;
                 tc_fence_after();
-                const uint32_t q = smem_u32(sQ + t * Cfg::TILE_BYTES), k = smem_u32(sK + s * Cfg::TILE_BYTES);
+                const uint32_t q = t ? q_lo1 : q_lo0, k = k_lo + s * (Cfg::TILE_BYTES >> 4);
+                const uint32_t dS = tS0 + t * 128;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
-                    umma_ss(tmem + Cfg::TMEM_S + t * 128, umma_desc_kmajor(q + off), umma_desc_kmajor(k + off), idescS,
-                            kk != 0);
+                    const uint32_t off = ((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
+                    umma_ss(dS, umma_desc_join(q + off, UMMA_DESC_HI_SW128), umma_desc_join(k + off, UMMA_DESC_HI_SW128),
+                            idescS, kk != 0);
                 }
                 umma_commit(&bars.s_full[t]);
                 if (t == last_t) umma_commit(&bars.k_empty[s]);
@@ -244,11 +253,19 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                 if (!mbar_wait(&bars.p_ready[t], j & 1, abortp)) return false;
                 if (!mbar_wait(&bars.v_full[s], (j / Cfg::VSTAGES) & 1, abortp)) return false;
                 tc_fence_after();
-                const uint32_t v = smem_u32(sV + s * Cfg::TILE_BYTES);
+                const uint32_t v = v_lo + s * (Cfg::TILE_BYTES >> 4);
+                const uint32_t dO = tO0 + t * D, aP = tS0 + t * 128;
+                if (j == 0) {
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    umma_ts(tmem + Cfg::TMEM_O + t * D, tmem + Cfg::TMEM_S + t * 128 + (kk >> 2) * 64 + (kk & 3) * 8,
-                            umma_desc_mnmajor(v + kk * 2048, 16384), idescO, (j | kk) != 0);
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(dO, aP + (kk >> 2) * 64 + (kk & 3) * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128),
+                                idescO, kk != 0);
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(dO, aP + (kk >> 2) * 64 + (kk & 3) * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128),
+                                idescO, 1);
+                }
                 umma_commit(&bars.o_done[t]);
                 if (t == last_t) umma_commit(&bars.v_empty[s]);
                 ++pv_blocks;
@@ -339,14 +356,17 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                 // ---- pass 2: P = exp2(S*sl2 - m) as bf16, stored over this thread's own half of S
                 // (columns [col_base, col_base + 32) of the block's TMEM region), behind its own reads.
                 float rowsum = 0.f;
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t v[32], pk[16];
-                    load32(c, v);
+                {
+                    uint32_t v0[32], v1[32], pk[16];
+                    load32(0, v0);
+                    load32(1, v1);
                     if (!SYM) tc_wait_ld();
-                    rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(v, sl2, -m_run, col_base + 32 * c, r, pk)
-                                   : exp_chunk32<Cfg::POLY_OF_4, false>(v, sl2, -m_run, col_base + 32 * c, r, pk);
-                    tmem_st16(tS + col_base + 16 * c, pk);
+                    rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(v0, sl2, -m_run, col_base, r, pk)
+                                   : exp_chunk32<Cfg::POLY_OF_4, false>(v0, sl2, -m_run, col_base, r, pk);
+                    tmem_st16(tS + col_base, pk);
+                    rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(v1, sl2, -m_run, col_base + 32, r, pk)
+                                   : exp_chunk32<Cfg::POLY_OF_4, false>(v1, sl2, -m_run, col_base + 32, r, pk);
+                    tmem_st16(tS + col_base + 16, pk);
                 }
                 l_run = fmaf(l_run, alpha, rowsum);
                 if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8

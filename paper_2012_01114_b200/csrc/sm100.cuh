@@ -174,6 +174,21 @@ __device__ __forceinline__ uint64_t umma_desc_kmajor(uint32_t saddr) { return um
 __device__ __forceinline__ uint64_t umma_desc_mnmajor(uint32_t saddr, uint32_t mn_block_bytes) {
     return umma_smem_desc(saddr, mn_block_bytes, 1024);
 }
+// Cheap descriptor arithmetic for the MMA-issuing thread.  The thread that issues tcgen05.mma is a
+// single lane; every instruction it spends per MMA delays the tensor pipe (a 128x128x16 MMA runs
+// for 64 cycles).  A descriptor is therefore split into its two 32-bit halves: the high half is a
+// constant of the layout, the low half is (address >> 4) | (leading offset field), so stepping the
+// start address by `bytes` (a multiple of 16, staying below 256 KB) is one 32-bit add of bytes >> 4.
+constexpr uint32_t UMMA_DESC_HI_SW128 = (1024u >> 4) | (1u << 14) | (UMMA_SWIZZLE_128B << 29);
+__device__ __forceinline__ uint32_t umma_desc_lo_kmajor(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t umma_desc_lo_mnmajor(uint32_t saddr, uint32_t mn_block_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | (((mn_block_bytes >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ uint64_t umma_desc_join(uint32_t lo, uint32_t hi) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
 // Instruction descriptor for kind::f16 with bf16 operands and fp32 accumulation.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(uint32_t M, uint32_t N, uint32_t a_major, uint32_t b_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (a_major << 15) | (b_major << 16) | ((N >> 3) << 17) |
