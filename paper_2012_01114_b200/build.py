@@ -35,7 +35,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + ".%d.tmp" % os.getpid()
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
            "--use_fast_math" if False else "-DPSA_BUILD", "-Xcompiler", "-fPIC,-O2", "-shared", "-cudart", "static",
-           "-o", tmp] + _sources()
+           "-o", tmp] + os.environ.get("PSA_NVCC_FLAGS", "").split() + _sources()
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
         print(" ".join(cmd))

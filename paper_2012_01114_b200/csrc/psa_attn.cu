@@ -16,10 +16,11 @@
 // kernel that computes one block per unordered tile pair and stores it at both mirror positions;
 // this kernel then runs phases 2 and 3 reading S from that scratch.
 //
-// CTA layout (576 threads): warp 0 = TMA producer, warp 1 = MMA issuer, warps 2-9 = softmax and
-// epilogue of row tile 0, warps 10-17 = the same for row tile 1.  Within a tile's eight warps, warp
-// pairs (w, w+4) share a TMEM lane quarter (32 rows) and split the 128 columns of S in halves; the
-// pair agrees on the row maximum through shared memory.  The two row tiles ping-pong: while the
+// CTA layout (576 threads with two softmax threads per row, the default): warp 0 = TMA producer, warp 1 =
+// MMA issuer, warps 2-9 = softmax and epilogue of row tile 0, warps 10-17 = the same for row tile 1.
+// Within a tile's eight warps, warp pairs (w, w+4) share a TMEM lane quarter (32 rows) and split the
+// 128 columns of S in halves; the pair agrees on the row maximum through shared memory.  (Built with
+// PSA_THREADS_PER_ROW=1 each row has one thread, four warps per tile, 320 threads.)  The two row tiles ping-pong: while the
 // softmax warps of one work on S_j, the tensor core runs the other's MMAs.
 // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [256+D,256+2D); P_t (bf16, two per column)
 // overlays S_t: keys 0-63 at S_t columns [0,32), keys 64-127 at [64,96), each written by the thread that
@@ -39,11 +40,18 @@ namespace psa {
 
 namespace {
 
+#ifndef PSA_RELOAD_S
+#define PSA_RELOAD_S 1
+#endif
 #ifndef PSA_POLY_OF_4
 #define PSA_POLY_OF_4 0
 #endif
 constexpr int CTRL_WARPS = 2;                       // producer, MMA issuer
-constexpr int SOFTMAX_WARPS_PER_TILE = 8;
+#ifndef PSA_THREADS_PER_ROW
+#define PSA_THREADS_PER_ROW 2
+#endif
+constexpr int TPR = PSA_THREADS_PER_ROW;            // softmax threads per query row (1 or 2)
+constexpr int SOFTMAX_WARPS_PER_TILE = 4 * TPR;
 constexpr int ATTN_THREADS = 32 * (CTRL_WARPS + 2 * SOFTMAX_WARPS_PER_TILE);   // 576
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float RESCALE_THRESHOLD = 8.0f;  // log2 units: O and l are rescaled only when the row max grew by more
@@ -231,11 +239,9 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
             const uint32_t k_lo = umma_desc_lo_kmajor(smem_u32(sK));
             const uint32_t v_lo = umma_desc_lo_mnmajor(smem_u32(sV), 16384);
             const uint32_t tS0 = tmem + Cfg::TMEM_S, tO0 = tmem + Cfg::TMEM_O;
-            auto issue_S = [&](int t, int j) -> bool {   // S_t = Q_t K_j^T        (phase 1, Eq. 1)
-                const int s = j % Cfg::KSTAGES;
-                if (!mbar_wait(&bars.k_full[s], (j / Cfg::KSTAGES) & 1, abortp)) return false;
-                tc_fence_after();
-                const uint32_t q = t ? q_lo1 : q_lo0, k = k_lo + s * (Cfg::TILE_BYTES >> 4);
+            // S_t = Q_t K_j^T (phase 1, Eq. 1): D/16 MMAs of 128x128x16 into the tile's S columns.
+            auto mma_S = [&](int t, int j) {
+                const uint32_t q = t ? q_lo1 : q_lo0, k = k_lo + (j % Cfg::KSTAGES) * (Cfg::TILE_BYTES >> 4);
                 const uint32_t dS = tS0 + t * 128;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
@@ -243,17 +249,19 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                     umma_ss(dS, umma_desc_join(q + off, UMMA_DESC_HI_SW128), umma_desc_join(k + off, UMMA_DESC_HI_SW128),
                             idescS, kk != 0);
                 }
-                umma_commit(&bars.s_full[t]);
-                if (t == last_t) umma_commit(&bars.k_empty[s]);
                 ++qk_blocks;
-                return true;
             };
-            auto issue_PV = [&](int t, int j) -> bool {  // O_t += P_t V_j         (phase 3, Eq. 3)
-                const int s = j % Cfg::VSTAGES;
+            // One step of one row tile: O_t += P_t V_j (phase 3, Eq. 3) and, when the tile has another key
+            // block, S_t for block j+1 right behind it (the tensor pipe runs them in order, so S may
+            // overwrite the columns P was read from).  One commit reports both to the softmax warps.
+            auto issue_step = [&](int t, int j, bool has_next) -> bool {
+                const int sv = j % Cfg::VSTAGES, sk = (j + 1) % Cfg::KSTAGES;
+                // operand tiles first: these are normally long complete and cost only the poll
+                if (!mbar_wait(&bars.v_full[sv], (j / Cfg::VSTAGES) & 1, abortp)) return false;
+                if (has_next && !mbar_wait(&bars.k_full[sk], ((j + 1) / Cfg::KSTAGES) & 1, abortp)) return false;
                 if (!mbar_wait(&bars.p_ready[t], j & 1, abortp)) return false;
-                if (!mbar_wait(&bars.v_full[s], (j / Cfg::VSTAGES) & 1, abortp)) return false;
                 tc_fence_after();
-                const uint32_t v = v_lo + s * (Cfg::TILE_BYTES >> 4);
+                const uint32_t v = v_lo + sv * (Cfg::TILE_BYTES >> 4);
                 const uint32_t dO = tO0 + t * D, aP = tS0 + t * 128;
                 if (j == 0) {
 #pragma unroll
@@ -266,20 +274,32 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                         umma_ts(dO, aP + (kk >> 2) * 64 + (kk & 3) * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128),
                                 idescO, 1);
                 }
-                umma_commit(&bars.o_done[t]);
-                if (t == last_t) umma_commit(&bars.v_empty[s]);
                 ++pv_blocks;
+                if (has_next) mma_S(t, j + 1);
+                umma_commit(&bars.o_done[t]);
+                if (t == last_t) {
+                    umma_commit(&bars.v_empty[sv]);
+                    if (has_next) umma_commit(&bars.k_empty[sk]);
+                }
                 return true;
             };
             for (int t = 0; t < work.ntiles && ok; ++t) ok = mbar_wait(&bars.q_full[t], 0, abortp);
-            if (!SYM)
-                for (int t = 0; t < work.ntiles && ok; ++t) ok = issue_S(t, 0);
-            for (int j = 0; j < maxkv && ok; ++j)
-                for (int t = 0; t < work.ntiles && ok; ++t)
-                    if (j < (t == 0 ? nkv0 : nkv1)) {
-                        ok = issue_PV(t, j);
-                        if (!SYM && ok && j + 1 < (t == 0 ? nkv0 : nkv1)) ok = issue_S(t, j + 1);
+            if (!SYM && ok) {
+                ok = mbar_wait(&bars.k_full[0], 0, abortp);
+                if (ok) {
+                    tc_fence_after();
+                    for (int t = 0; t < work.ntiles; ++t) {
+                        mma_S(t, 0);
+                        umma_commit(&bars.s_full[t]);
                     }
+                    umma_commit(&bars.k_empty[0]);
+                }
+            }
+            for (int j = 0; j < maxkv && ok; ++j)
+                for (int t = 0; t < work.ntiles && ok; ++t) {
+                    const int nkv_t = t == 0 ? nkv0 : nkv1;
+                    if (j < nkv_t) ok = issue_step(t, j, !SYM && j + 1 < nkv_t);
+                }
             const unsigned long long block_macs = (unsigned long long)TILE * TILE * D;
             if (qk_blocks) atomicAdd(&dc->qk_macs, qk_blocks * block_macs);
             if (pv_blocks) {
@@ -289,30 +309,36 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
         }
     } else {
         // ------------------------------------------------------------ softmax + epilogue
+        // TPR threads share a query row; thread `part` owns block columns [part*CPT, (part+1)*CPT).
+        constexpr int CPT = 128 / TPR;                           // score columns per thread
+        constexpr int NCH = CPT / 32;                            // 32-column chunks per thread
+        constexpr int OPT = D / TPR;                             // output columns per thread
         const int sw = warp - CTRL_WARPS;
-        const int t = sw >> 3;                                  // row tile of this warp
-        const int hlf = (sw >> 2) & 1;                          // column half of S / O this thread owns
+        const int t = sw / SOFTMAX_WARPS_PER_TILE;              // row tile of this warp
+        const int part = (sw % SOFTMAX_WARPS_PER_TILE) >> 2;    // which share of the row's columns
         const int nkv = t == 0 ? nkv0 : nkv1;
         if (t < work.ntiles) {
             const int q = warp & 3;                             // TMEM lane quarter this warp may access
             const int r = q * 32 + lane;                        // row inside the tile = TMEM lane
             const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
             const uint32_t tS = tmem + Cfg::TMEM_S + t * 128 + lane_off;
-            const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off + hlf * (D / 2);
+            const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off + part * OPT;
             const int It = work.tile0 + t;
-            const int pair_bar = 1 + t * 4 + q;                 // named barrier of the two warps sharing rows
-            const int tile_bar = 9 + t;                         // named barrier of the tile's eight warps
-            const int col_base = hlf * 64;
+            const int pair_bar = 1 + t * 4 + q;                 // named barrier of the warps sharing rows
+            const int tile_bar = 9 + t;                         // named barrier of all softmax warps of the tile
+            const int col_base = part * CPT;
             const float* srow = SYM ? Sg + ((size_t)work.bh * n + (size_t)It * TILE + r) * n + col_base : nullptr;
             float m_run = -INFINITY, l_run = 0.f;
             bool ok = true;
             for (int j = 0; j < nkv; ++j) {
-                if (!SYM) ok = mbar_wait(&bars.s_full[t], j & 1, abortp);
-                if (ok && j > 0) ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);  // PV_{j-1} done with P and O
+                // block 0 waits for the first S; later blocks for the commit that follows PV_{j-1} and S_j
+                if (j == 0) { if (!SYM) ok = mbar_wait(&bars.s_full[t], 0, abortp); }
+                else ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);
                 ok = __all_sync(0xffffffffu, ok);
+                if (TPR == 1 && !ok) break;
                 const bool diag = (scheme == PSA_MASKED) && (j == It);
                 float mx = -INFINITY;
-                // 32 raw scores of this thread's half row: chunk c covers block columns col_base + 32c ..
+                // 32 raw scores of this thread's share of the row: chunk c = block columns col_base + 32c ..
                 auto load32 = [&](int c, uint32_t (&v)[32]) {
                     if (!SYM) {
                         tmem_ld32(tS + col_base + 32 * c, v);
@@ -326,52 +352,52 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                         }
                     }
                 };
+                uint32_t sreg[NCH][32];
                 if (ok) {
-                    // ---- pass 1: maximum of this thread's 64 scores
+                    // ---- pass 1: maximum of this thread's scores
                     tc_fence_after();
-                    uint32_t a[32], bb[32];
-                    load32(0, a);
-                    load32(1, bb);
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) load32(c, sreg[c]);
                     if (!SYM) tc_wait_ld();
-                    if (diag) {
-                        mx = max_chunk32<true>(a, col_base, r, mx);
-                        mx = max_chunk32<true>(bb, col_base + 32, r, mx);
-                    } else {
-                        mx = max_chunk32<false>(a, col_base, r, mx);
-                        mx = max_chunk32<false>(bb, col_base + 32, r, mx);
-                    }
-                    xch_max[j & 1][t][hlf][r] = mx;
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c)
+                        mx = diag ? max_chunk32<true>(sreg[c], col_base + 32 * c, r, mx)
+                                  : max_chunk32<false>(sreg[c], col_base + 32 * c, r, mx);
                 }
-                // The two threads of a row meet here to exchange their half-row maxima (and to leave
-                // together if either gave up a wait).
-                ok = named_bar_all(ok, pair_bar, 64);
-                if (!ok) break;
-                mx = fmaxf(mx, xch_max[j & 1][t][hlf ^ 1][r]);
+                if (TPR == 2) {
+                    // The two threads of a row meet here to exchange their half-row maxima (and to leave
+                    // together if either gave up a wait).
+                    xch_max[j & 1][t][part][r] = mx;
+                    ok = named_bar_all(ok, pair_bar, 64);
+                    if (!ok) break;
+                    mx = fmaxf(mx, xch_max[j & 1][t][part ^ 1][r]);
+                }
                 const float mx2 = mx * sl2;
                 float alpha = 1.f;
                 if (mx2 > m_run + RESCALE_THRESHOLD) {   // also taken on the first block (m_run = -inf)
                     alpha = ex2_mufu(m_run - mx2);
                     m_run = mx2;
                 }
-                // ---- pass 2: P = exp2(S*sl2 - m) as bf16, stored over this thread's own half of S
-                // (columns [col_base, col_base + 32) of the block's TMEM region), behind its own reads.
+                // ---- pass 2: P = exp2(S*sl2 - m) as bf16, stored over this thread's own share of S, behind
+                // its own reads: keys [col_base + 32c, +32) go to S columns (col_base/64)*64 + (col_base%64)/2 + 16c.
                 float rowsum = 0.f;
-                {
-                    uint32_t v0[32], v1[32], pk[16];
-                    load32(0, v0);
-                    load32(1, v1);
+                if (TPR == 2 && PSA_RELOAD_S) {
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) load32(c, sreg[c]);
                     if (!SYM) tc_wait_ld();
-                    rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(v0, sl2, -m_run, col_base, r, pk)
-                                   : exp_chunk32<Cfg::POLY_OF_4, false>(v0, sl2, -m_run, col_base, r, pk);
-                    tmem_st16(tS + col_base, pk);
-                    rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(v1, sl2, -m_run, col_base + 32, r, pk)
-                                   : exp_chunk32<Cfg::POLY_OF_4, false>(v1, sl2, -m_run, col_base + 32, r, pk);
-                    tmem_st16(tS + col_base + 16, pk);
+                }
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    uint32_t pk[16];
+                    const int kc = col_base + 32 * c;            // first key column of the chunk
+                    rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(sreg[c], sl2, -m_run, kc, r, pk)
+                                   : exp_chunk32<Cfg::POLY_OF_4, false>(sreg[c], sl2, -m_run, kc, r, pk);
+                    tmem_st16(tS + (kc >> 6) * 64 + ((kc & 63) >> 1), pk);
                 }
                 l_run = fmaf(l_run, alpha, rowsum);
                 if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8
 #pragma unroll
-                    for (int c = 0; c < D / 64; ++c) {
+                    for (int c = 0; c < OPT / 32; ++c) {
                         uint32_t v[32];
                         tmem_ld32(tO + 32 * c, v);
                         tc_wait_ld();
@@ -385,15 +411,15 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                 mbar_arrive(&bars.p_ready[t]);
             }
             if (ok) ok = mbar_wait(&bars.o_done[t], (nkv - 1) & 1, abortp);
-            xch_sum[t][hlf][r] = l_run;
+            if (TPR == 2) xch_sum[t][part][r] = l_run;
             if (named_bar_all(ok, tile_bar, 32 * SOFTMAX_WARPS_PER_TILE)) {
                 // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row)
                 tc_fence_after();
-                const float inv = 1.f / (l_run + xch_sum[t][hlf ^ 1][r]);
+                const float inv = 1.f / (TPR == 2 ? l_run + xch_sum[t][part ^ 1][r] : l_run);
                 uint8_t* stage = sQ + t * Cfg::TILE_BYTES;     // Q_t is no longer read by any MMA
 #pragma unroll
-                for (int c = 0; c < D / 64; ++c) {
-                    const int col = hlf * (D / 2) + 32 * c;    // first of 32 output columns handled here
+                for (int c = 0; c < OPT / 32; ++c) {
+                    const int col = part * OPT + 32 * c;       // first of 32 output columns handled here
                     uint32_t v[32];
                     tmem_ld32(tO + 32 * c, v);
                     tc_wait_ld();
@@ -410,7 +436,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                 }
                 fence_async_smem();
                 named_bar_sync(tile_bar, 32 * SOFTMAX_WARPS_PER_TILE);
-                if (sw == t * 8 && lane == 0) {
+                if (sw == t * SOFTMAX_WARPS_PER_TILE && lane == 0) {
                     for (int u = 0; u < Cfg::SUB; ++u)
                         tma_store_2d(&maps.o, stage + u * 16384, col0 + 64 * u, row0 + It * TILE);
                     tma_store_commit();

@@ -53,14 +53,19 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                  : "memory");
 }
+// One poll; the hardware may park the thread for up to PSA_TRY_WAIT_HINT_NS while the phase is pending,
+// which keeps waiting warps out of the issue slots of the warps that are working.
+#ifndef PSA_TRY_WAIT_HINT_NS
+#define PSA_TRY_WAIT_HINT_NS 100000u
+#endif
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(PSA_TRY_WAIT_HINT_NS)
         : "memory");
     return ok != 0;
 }
