@@ -29,20 +29,33 @@ def _mix64(x: np.ndarray) -> np.ndarray:
         return x ^ (x >> np.uint64(31))
 
 
+def _normal_chunk(key, lo, hi, out, base):
+    k = np.arange(lo, hi, dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        a = _mix64(key ^ (k * np.uint64(2)))
+        b = _mix64(key ^ (k * np.uint64(2) + np.uint64(1)))
+    u1 = ((a >> np.uint64(11)).astype(np.float64) + 0.5) * (1.0 / 9007199254740992.0)
+    u2 = ((b >> np.uint64(11)).astype(np.float64) + 0.5) * (1.0 / 9007199254740992.0)
+    out[lo - base:hi - base] = np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
+
+
 def normal(seed: int, tensor_id: int, count: int, start: int = 0) -> np.ndarray:
-    """`count` standard-normal float64 draws for elements start .. start+count-1 of a tensor."""
+    """`count` standard-normal float64 draws for elements start .. start+count-1 of a tensor.
+
+    Element k depends on (seed, tensor_id, k) only; large requests are drawn in chunks on a thread pool
+    (numpy releases the GIL inside its loops), which changes nothing about the values."""
     out = np.empty(count, dtype=np.float64)
     key = _mix64(np.array([np.uint64(seed) * np.uint64(0x100000001B3) + np.uint64(tensor_id)], dtype=np.uint64))[0]
-    step = 1 << 22
-    for lo in range(0, count, step):
-        hi = min(count, lo + step)
-        k = np.arange(start + lo, start + hi, dtype=np.uint64)
-        with np.errstate(over="ignore"):
-            a = _mix64(key ^ (k * np.uint64(2)))
-            b = _mix64(key ^ (k * np.uint64(2) + np.uint64(1)))
-        u1 = ((a >> np.uint64(11)).astype(np.float64) + 0.5) * (1.0 / 9007199254740992.0)
-        u2 = ((b >> np.uint64(11)).astype(np.float64) + 0.5) * (1.0 / 9007199254740992.0)
-        out[lo:hi] = np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
+    step = 1 << 20
+    spans = [(start + lo, start + min(count, lo + step)) for lo in range(0, count, step)]
+    if len(spans) <= 2:
+        for lo, hi in spans:
+            _normal_chunk(key, lo, hi, out, start)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        import os
+        with ThreadPoolExecutor(max_workers=min(32, os.cpu_count() or 1)) as ex:
+            list(ex.map(lambda sp: _normal_chunk(key, sp[0], sp[1], out, start), spans))
     return out
 
 
@@ -71,6 +84,17 @@ def tensor(seed: int, tensor_id: int, shape, scale: float, dtype: str):
         f = x.astype(np.float32).reshape(shape)
         return f.astype(np.float64), f
     raise ValueError(dtype)
+
+
+def tensor_bits(seed: int, tensor_id: int, shape, scale: float) -> np.ndarray:
+    """bf16 bit patterns only (for tensors too large to also keep as float64); same numbers as `tensor`."""
+    count = int(np.prod(shape))
+    out = np.empty(count, dtype=np.uint16)
+    step = 1 << 24
+    for lo in range(0, count, step):
+        hi = min(count, lo + step)
+        out[lo:hi] = to_bf16_bits(normal(seed, tensor_id, hi - lo, start=lo) * scale)
+    return out.reshape(shape)
 
 
 # The five workloads (shape, number type, scheme, seed).  `proj` says whether X and the three
