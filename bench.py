@@ -167,6 +167,67 @@ def config_of(w, args):
             "l2": "flushed between steps by an untimed %d MiB memset" % (L2_FLUSH_BYTES >> 20)}
 
 
+def run_sweep(args):
+    """Workload family c5: n in {256, 1024, 4096, 16384} x {full, symmetric, masked}, 16 heads x 128, batch*n =
+    65536 tokens, core only.  One JSON line: per point the time, useful TFLOP/s, measured issued fraction and the
+    wall-time ratio against the same size computed without skipping."""
+    import torch
+    from paper_2012_01114_b200 import binding as psa, build, inputs
+    build.build()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    peaks = measured_peaks()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    points = []
+    for n in (256, 1024, 4096, 16384):
+        w0 = inputs.WORKLOADS["c5-n%d-full" % n]
+        B, H, d = w0["batch"], w0["heads"], w0["d_k"]
+        dev = {k: torch.from_numpy(inputs.tensor_bits(w0["seed"], t, (B, n, H, d), 1.0).view(np.int16)).cuda().view(torch.bfloat16)
+               for k, t in (("Q", 4), ("K", 5), ("V", 6))}
+        out = torch.empty((B, n, H * d), dtype=torch.bfloat16, device="cuda")
+        t_full = None
+        for scheme in (psa.FULL, psa.SYMMETRIC, psa.MASKED):
+            w = dict(inputs.WORKLOADS["c5-n%d-%s" % (n, inputs.SCHEME_NAMES[scheme])])
+            sym = scheme == psa.SYMMETRIC
+
+            def step():
+                psa.psa_attention_core(dev["Q"], None if sym else dev["K"], None if sym else dev["V"], scheme, out=out)
+            for _ in range(max(3, args.warmup)):
+                flush.zero_(); step()
+            torch.cuda.synchronize()
+            st, issued = psa.psa_last_issued()
+            if st != psa.OK:
+                raise RuntimeError("device status %d" % st)
+            steps = max(5, min(args.steps, 20))
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+            for a, b in ev:
+                flush.zero_(); a.record(); step(); b.record()
+            torch.cuda.synchronize()
+            ms = sorted(a.elapsed_time(b) for a, b in ev)
+            med = ms[len(ms) // 2]
+            fl = useful_flops(w)["core"]
+            full_macs = 2.0 * B * H * d * n * n
+            if scheme == psa.FULL:
+                t_full = med
+            bytes_alg = (2 if sym else 4) * B * n * H * d * 2
+            points.append({"n": n, "batch": B, "scheme": inputs.SCHEME_NAMES[scheme], "ms": med, "ms_min": ms[0],
+                           "useful_tflops": fl / (med * 1e-3) / 1e12,
+                           "pct_of_measured_bf16_peak": 100.0 * fl / (med * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                           "algorithmic_gbs": bytes_alg / (med * 1e-3) / 1e9,
+                           "pct_of_measured_hbm": 100.0 * bytes_alg / (med * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                           "issued_macs": issued["qk_macs"] + issued["pv_macs"],
+                           "useful_macs": issued["useful_qk_macs"] + issued["useful_pv_macs"],
+                           "issued_fraction_of_full": (issued["qk_macs"] + issued["pv_macs"]) / full_macs,
+                           "useful_fraction_of_full": (issued["useful_qk_macs"] + issued["useful_pv_macs"]) / full_macs,
+                           "time_ratio_full_over_scheme": (t_full / med) if t_full else None})
+        del dev, out
+    best = max((p for p in points if p["scheme"] == "masked"), key=lambda p: p["useful_tflops"])
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "value": best["useful_tflops"], "n_gpus": 1, "dtype": "bf16",
+                      "data": "synthetic", "higher_is_better": True,
+                      "config": {"workload": "c5 sweep (value = best masked point, n=%d)" % best["n"],
+                                 "l2": "flushed between steps by an untimed %d MiB memset" % (L2_FLUSH_BYTES >> 20)},
+                      "peaks": peaks, "sweep": points}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -174,6 +235,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--impl", default="psa", choices=["psa", "reference"])
+    ap.add_argument("--sweep", action="store_true", help="time the twelve points of workload family c5 (one JSON line)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer pass (for profiler captures)")
     args = ap.parse_args()
@@ -184,6 +246,10 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
     from paper_2012_01114_b200 import inputs
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args)
+        return 0
     if args.impl == "reference":
         if rank == 0:
             w = dict(inputs.WORKLOADS[args.workload]); w["name"] = args.workload
