@@ -116,17 +116,27 @@ gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, Dev
     } else if (warp == 1 && lane == 0) {
         // ---- MMA issuer
         const uint32_t idesc = umma_idesc_bf16(BM, BN, UMMA_K_MAJOR, UMMA_MN_MAJOR);
+        // descriptor low words of stage 0; a stage or k-step is a constant added to them (sm100.cuh)
+        const uint32_t a_lo0 = umma_desc_lo_kmajor(smem_u32(smem));
+        const uint32_t b_lo0 = umma_desc_lo_mnmajor(smem_u32(smem + A_BYTES), B_SUB_BYTES);
         bool ok = true;
         for (int kt = 0; kt < nk && ok; ++kt) {
             const int s = kt % STAGES;
             ok = mbar_wait(&full_bar[s], (kt / STAGES) & 1, abortp);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t sA = smem_u32(smem + s * STAGE_BYTES), sB = sA + A_BYTES;
+            const uint32_t a_lo = a_lo0 + s * (STAGE_BYTES >> 4), b_lo = b_lo0 + s * (STAGE_BYTES >> 4);
+            if (kt == 0) {
 #pragma unroll
-            for (int k = 0; k < BK / 16; ++k)
-                umma_ss(tmem, umma_desc_kmajor(sA + k * 32), umma_desc_mnmajor(sB + k * 2048, B_SUB_BYTES), idesc,
-                        (kt | k) != 0);
+                for (int k = 0; k < BK / 16; ++k)
+                    umma_ss(tmem, umma_desc_join(a_lo + k * (32 >> 4), UMMA_DESC_HI_SW128),
+                            umma_desc_join(b_lo + k * (2048 >> 4), UMMA_DESC_HI_SW128), idesc, k != 0);
+            } else {
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    umma_ss(tmem, umma_desc_join(a_lo + k * (32 >> 4), UMMA_DESC_HI_SW128),
+                            umma_desc_join(b_lo + k * (2048 >> 4), UMMA_DESC_HI_SW128), idesc, 1);
+            }
             umma_commit(&empty_bar[s]);
         }
         if (ok) {
