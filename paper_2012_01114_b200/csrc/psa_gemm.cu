@@ -1,8 +1,8 @@
 // Projection GEMM for the bf16 path (paper Sec. 3.1: q, k, v = x*Wq, x*Wk, x*Wv):
 //     C_w[M, N] = A[M, K] * B_w[K, N],  w < nW,  bf16 row-major operands, fp32 accumulation in TMEM.
 //
-// One CTA per 128x128 output tile (two CTAs resident per SM so one tile's epilogue overlaps the
-// other's main loop).  Warp 0 streams operand tiles with TMA into a 3-stage shared-memory ring,
+// One CTA per 128 x BN output tile (BN = 256; two CTAs resident per SM so one tile's epilogue overlaps
+// the other's main loop).  Warp 0 streams operand tiles with TMA into a shared-memory ring,
 // warp 1 issues tcgen05 MMAs (A K-major, B in its natural row-major form = MN-major), warps 2-5
 // move the accumulator TMEM -> registers -> bf16 -> swizzled shared memory -> TMA store.
 #include <stdio.h>
@@ -52,12 +52,20 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uin
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64;
-constexpr int STAGES = 3;
+#ifndef PSA_GEMM_BN
+#define PSA_GEMM_BN 256
+#endif
+#ifndef PSA_GEMM_STAGES
+#define PSA_GEMM_STAGES 2
+#endif
+constexpr int BM = 128, BN = PSA_GEMM_BN, BK = 64;
+constexpr int NSUB = BN / 64;                  // 64-column sub-tiles of B and C per tile
+constexpr int STAGES = PSA_GEMM_STAGES;
 constexpr int A_BYTES = BM * BK * 2;           // 16 KB, K-major [128 x 64]
 constexpr int B_SUB_BYTES = BK * 64 * 2;       // 8 KB, one [64 k-rows x 64 n] sub-tile
-constexpr int B_BYTES = 2 * B_SUB_BYTES;       // 16 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES; // 32 KB
+constexpr int B_BYTES = NSUB * B_SUB_BYTES;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+static_assert(STAGES * STAGE_BYTES >= BM * BN * 2, "the drained ring doubles as the output staging buffer");
 constexpr int GEMM_THREADS = 192;
 constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024;  // + slack for 1024-byte alignment
 
@@ -105,8 +113,8 @@ gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, Dev
             uint8_t* sB = sA + A_BYTES;
             mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
             tma_load_2d(sA, &maps.a, &full_bar[s], kt * BK, m0);
-            tma_load_2d(sB, mapB, &full_bar[s], n0, kt * BK);
-            tma_load_2d(sB + B_SUB_BYTES, mapB, &full_bar[s], n0 + 64, kt * BK);
+#pragma unroll
+            for (int u = 0; u < NSUB; ++u) tma_load_2d(sB + u * B_SUB_BYTES, mapB, &full_bar[s], n0 + 64 * u, kt * BK);
             ++issued;
         }
         if (*abortp) {  // let copies already in flight land before the CTA goes away
@@ -171,8 +179,9 @@ gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, Dev
             fence_async_smem();
             named_bar_sync(1, 128);
             if (warp == 2 && lane == 0) {
-                tma_store_2d(mapC, stage, n0, m0);
-                if (n0 + 64 < N) tma_store_2d(mapC, stage + BM * 128, n0 + 64, m0);
+#pragma unroll
+                for (int u = 0; u < NSUB; ++u)
+                    if (n0 + 64 * u < N) tma_store_2d(mapC, stage + u * (BM * 128), n0 + 64 * u, m0);
                 tma_store_commit();
                 tma_store_wait_all();
             }
