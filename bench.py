@@ -37,6 +37,40 @@ UNIT = "TFLOP/s"
 L2_FLUSH_BYTES = 256 << 20
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
+# (attn_kernel_c4_masked_n8192_d128.txt, gemm_and_attn_c3_masked_n1024_d64.txt).  Each figure is tied to the
+# SHA-256 of the kernel source it was measured on; once that source changes the roofline reports traffic = null.
+NCU_TRAFFIC = {
+    "sources": {
+        "attn": "fc68ce3e412a2c975dab5b3bbdf04c41081304e49a19d22d2f6693d69ddf062a",
+        "proj": "a0e3018c778ef73c0e369cb34617797055238c0b7013d90d881b6e8f2572c6cf",
+        "common": "f4c4c8e46254e54a9901d3bf7409741f97e645a86bd07fcca32545538100330c"
+    },
+    "traffic_bytes": {
+        "c4": {
+            "attn": 251813632
+        },
+        "c3": {
+            "attn": 37849856,
+            "proj": 16195328
+        }
+    }
+}
+
+
+def ncu_traffic(workload, kernel):
+    import hashlib
+    files = {"attn": "psa_attn.cu", "proj": "psa_gemm.cu", "common": "sm100.cuh"}
+    try:
+        for key in (kernel, "common"):
+            with open(os.path.join(ROOT, "paper_2012_01114_b200", "csrc", files[key]), "rb") as f:
+                if hashlib.sha256(f.read()).hexdigest() != NCU_TRAFFIC["sources"][key]:
+                    return None
+        return NCU_TRAFFIC["traffic_bytes"].get(workload, {}).get(kernel)
+    except OSError:
+        return None
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -384,7 +418,8 @@ def main():
     roofline = {"bound": "tensor", "kernel": "attn_kernel (fused scores-softmax-weighted sum)" if dominant == "attn" else "gemm_bf16_kernel (projections)",
                 "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": (achieved / peaks["bf16_tflops"]) if achieved else None, "peak_source": peaks["source"] + " burst bf16",
-                "traffic": None, "kernel_ms": kern, "algorithmic_flops": alg,
+                "traffic": ncu_traffic(args.workload, dominant), "traffic_unit": "bytes per launch (ncu)",
+                "kernel_ms": kern, "algorithmic_flops": alg,
                 "issued_flops": issued_flops}
     cpu = None
     if not args.no_cpu_baseline and world == 1:
