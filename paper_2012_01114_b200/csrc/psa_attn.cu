@@ -381,7 +381,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                 // ---- pass 2: P = exp2(S*sl2 - m) as bf16, stored over this thread's own share of S, behind
                 // its own reads: keys [col_base + 32c, +32) go to S columns (col_base/64)*64 + (col_base%64)/2 + 16c.
                 float rowsum = 0.f;
-                if (TPR == 2 && PSA_RELOAD_S) {
+                if (TPR == 2 && PSA_RELOAD_S) {      // the scores were only reduced so far: fetch them again
 #pragma unroll
                     for (int c = 0; c < NCH; ++c) load32(c, sreg[c]);
                     if (!SYM) tc_wait_ld();
@@ -440,7 +440,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                     for (int u = 0; u < Cfg::SUB; ++u)
                         tma_store_2d(&maps.o, stage + u * 16384, col0 + 64 * u, row0 + It * TILE);
                     tma_store_commit();
-                    tma_store_wait_all();
+                    tma_store_wait_read();   // smem may be released; the writes complete on their own
                 }
             }
         }
