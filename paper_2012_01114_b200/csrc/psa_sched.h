@@ -30,19 +30,34 @@ struct CtaWork {
 PSA_HD int row_tiles(int n) { return n / TILE; }
 PSA_HD int ctas_per_head(int n) { return (row_tiles(n) + TILES_PER_CTA - 1) / TILES_PER_CTA; }
 
-// CTA index -> work.  Heads are the slow index so that CTAs resident together read the same K and
-// V (L2 reuse); inside a head the masked scheme hands out the heaviest row tiles first (the role of
-// the paper's pairing of long rows with short ones, Sec. 5.2: balance).
-PSA_HD CtaWork cta_work(int cta, int n, int scheme_masked) {
+// CTA index -> work, for a launch over `nbh` (batch, head) units.
+//   head-major order (global_lpt = 0): heads are the slow index so that CTAs resident together read the
+//     same K and V (L2 reuse); inside a head the masked scheme hands out the heaviest row tiles first.
+//   global order (global_lpt = 1, masked scheme on problems whose K and V all fit in L2 anyway): all heads'
+//     heaviest row-tile pairs first, then the next heaviest, ... so that the hardware's in-order CTA
+//     dispatch amounts to longest-processing-time-first scheduling.
+// Both play the role of the paper's pairing of long rows with short ones (Sec. 5.2): balance.
+PSA_HD CtaWork cta_work(int cta, int n, int scheme_masked, int nbh, int global_lpt) {
     const int P = ctas_per_head(n);
     CtaWork w;
-    w.bh = cta / P;
-    const int r = cta - w.bh * P;
+    int r;
+    if (global_lpt) {
+        r = cta / nbh;
+        w.bh = cta - r * nbh;
+    } else {
+        w.bh = cta / P;
+        r = cta - w.bh * P;
+    }
     const int p = scheme_masked ? (P - 1 - r) : r;
     w.tile0 = p * TILES_PER_CTA;
     const int left = row_tiles(n) - w.tile0;
     w.ntiles = left < TILES_PER_CTA ? left : TILES_PER_CTA;
     return w;
+}
+// Whether a masked launch uses the global order: K and V of every head together stay below this many bytes.
+constexpr long long GLOBAL_LPT_MAX_KV_BYTES = 48ll << 20;
+PSA_HD int use_global_lpt(int scheme, long long nbh, int n, int d) {
+    return scheme == PSA_MASKED && nbh * n * d * 2 * 2 <= GLOBAL_LPT_MAX_KV_BYTES;
 }
 
 // Number of key/value tiles row tile I visits in phases 1-3 of the fused kernel (FULL, MASKED) or
