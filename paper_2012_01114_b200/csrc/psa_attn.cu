@@ -170,6 +170,26 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
     const int maxkv = max(nkv0, nkv1);
     const int last_t = work.ntiles - 1;
 
+    // TMA requests of one Q, K or V tile (issued by thread 0 only)
+    auto load_q = [&](int t) {
+        mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
+        for (int u = 0; u < Cfg::SUB; ++u)
+            tma_load_2d(sQ + t * Cfg::TILE_BYTES + u * 16384, &maps.q, &bars.q_full[t], col0 + 64 * u,
+                        row0 + (work.tile0 + t) * TILE);
+    };
+    auto load_k = [&](int j) {
+        if (SYM) return;
+        const int s = j % Cfg::KSTAGES;
+        mbar_arrive_expect_tx(&bars.k_full[s], Cfg::TILE_BYTES);
+        for (int u = 0; u < Cfg::SUB; ++u)
+            tma_load_2d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], col0 + 64 * u, row0 + j * TILE);
+    };
+    auto load_v = [&](int j) {
+        const int s = j % Cfg::VSTAGES;
+        mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
+        for (int u = 0; u < Cfg::SUB; ++u)
+            tma_load_2d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], col0 + 64 * u, row0 + j * TILE);
+    };
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int t = 0; t < 2; ++t) {
@@ -183,8 +203,13 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
             mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], 1);
         }
         fence_mbar_init();
+        // The first operand tiles need no free-stage wait: request them now, so that their flight
+        // overlaps the TMEM allocation and the CTA-wide barrier below.
+        for (int t = 0; t < work.ntiles; ++t) load_q(t);
+        for (int j = 0; j < maxkv && j < Cfg::KSTAGES; ++j) load_k(j);
+        for (int j = 0; j < maxkv && j < Cfg::VSTAGES; ++j) load_v(j);
     }
-    if (warp == 0) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
+    if (warp == 1) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -194,30 +219,19 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
     if (warp == 0) {
         if (lane == 0) {
             // ------------------------------------------------------------ TMA producer
-            for (int t = 0; t < work.ntiles; ++t) {
-                mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
-                for (int s = 0; s < Cfg::SUB; ++s)
-                    tma_load_2d(sQ + t * Cfg::TILE_BYTES + s * 16384, &maps.q, &bars.q_full[t], col0 + 64 * s,
-                                row0 + (work.tile0 + t) * TILE);
-            }
-            int jk = 0, jv = 0;
+            // (Q and the first KSTAGES / VSTAGES key and value tiles were requested during set-up.)
+            int jk = SYM ? 0 : min(maxkv, Cfg::KSTAGES), jv = min(maxkv, Cfg::VSTAGES);
             for (int j = 0; j < maxkv; ++j) {
-                if (!SYM) {
-                    const int s = j % Cfg::KSTAGES;
-                    if (j >= Cfg::KSTAGES && !mbar_wait(&bars.k_empty[s], ((j / Cfg::KSTAGES) - 1) & 1, abortp)) break;
-                    mbar_arrive_expect_tx(&bars.k_full[s], Cfg::TILE_BYTES);
-                    for (int u = 0; u < Cfg::SUB; ++u)
-                        tma_load_2d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], col0 + 64 * u,
-                                    row0 + j * TILE);
+                if (!SYM && j >= Cfg::KSTAGES) {
+                    if (!mbar_wait(&bars.k_empty[j % Cfg::KSTAGES], ((j / Cfg::KSTAGES) - 1) & 1, abortp)) break;
+                    load_k(j);
                     jk = j + 1;
                 }
-                const int s = j % Cfg::VSTAGES;
-                if (j >= Cfg::VSTAGES && !mbar_wait(&bars.v_empty[s], ((j / Cfg::VSTAGES) - 1) & 1, abortp)) break;
-                mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
-                for (int u = 0; u < Cfg::SUB; ++u)
-                    tma_load_2d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], col0 + 64 * u,
-                                row0 + j * TILE);
-                jv = j + 1;
+                if (j >= Cfg::VSTAGES) {
+                    if (!mbar_wait(&bars.v_empty[j % Cfg::VSTAGES], ((j / Cfg::VSTAGES) - 1) & 1, abortp)) break;
+                    load_v(j);
+                    jv = j + 1;
+                }
             }
             if (*abortp) {  // let copies already issued land before shared memory is released
                 for (int t = 0; t < work.ntiles; ++t) mbar_wait_drain(&bars.q_full[t], 0);
@@ -448,7 +462,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && abort_flag) atomicExch(&dc->status, (int)PSA_ERR_TIMEOUT);
-    if (warp == 0) tmem_dealloc(tmem, 512);
+    if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
 
