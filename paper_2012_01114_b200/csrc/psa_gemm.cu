@@ -1,10 +1,11 @@
 // Projection GEMM for the bf16 path (paper Sec. 3.1: q, k, v = x*Wq, x*Wk, x*Wv):
 //     C_w[M, N] = A[M, K] * B_w[K, N],  w < nW,  bf16 row-major operands, fp32 accumulation in TMEM.
 //
-// One CTA per 128 x BN output tile (BN = 256; two CTAs resident per SM so one tile's epilogue overlaps
-// the other's main loop).  Warp 0 streams operand tiles with TMA into a shared-memory ring,
-// warp 1 issues tcgen05 MMAs (A K-major, B in its natural row-major form = MN-major), warps 2-5
-// move the accumulator TMEM -> registers -> bf16 -> swizzled shared memory -> TMA store.
+// Persistent kernel, one CTA per SM, walking 128 x 256 output tiles (all three weight matrices in one
+// launch).  Warp 0 streams operand tiles with TMA into a shared-memory ring, warp 1 issues tcgen05 MMAs
+// (A K-major, B in its natural row-major form = MN-major) into one of two 256-column TMEM accumulators,
+// warps 2-5 drain the other accumulator (TMEM -> registers -> bf16 -> swizzled shared memory -> TMA
+// store), so that a tile's epilogue runs under the next tile's main loop.
 #include <stdio.h>
 
 #include <mutex>
@@ -52,22 +53,21 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uin
 
 namespace {
 
-#ifndef PSA_GEMM_BN
-#define PSA_GEMM_BN 256
-#endif
-#ifndef PSA_GEMM_STAGES
-#define PSA_GEMM_STAGES 2
-#endif
-constexpr int BM = 128, BN = PSA_GEMM_BN, BK = 64;
+constexpr int BM = 128, BN = 256, BK = 64;
 constexpr int NSUB = BN / 64;                  // 64-column sub-tiles of B and C per tile
+#ifndef PSA_GEMM_STAGES
+#define PSA_GEMM_STAGES 4
+#endif
 constexpr int STAGES = PSA_GEMM_STAGES;
 constexpr int A_BYTES = BM * BK * 2;           // 16 KB, K-major [128 x 64]
 constexpr int B_SUB_BYTES = BK * 64 * 2;       // 8 KB, one [64 k-rows x 64 n] sub-tile
-constexpr int B_BYTES = NSUB * B_SUB_BYTES;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-static_assert(STAGES * STAGE_BYTES >= BM * BN * 2, "the drained ring doubles as the output staging buffer");
+constexpr int B_BYTES = NSUB * B_SUB_BYTES;    // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES; // 48 KB
+constexpr int OUT_COLS = 128;                  // the epilogue moves a tile out in column halves
+constexpr int OUT_BYTES = BM * OUT_COLS * 2;   // 32 KB output staging (two swizzled [128 x 64] sub-tiles)
 constexpr int GEMM_THREADS = 192;
-constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024;  // + slack for 1024-byte alignment
+constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + OUT_BYTES + 1024;  // + slack for 1024-byte alignment
+constexpr int TMEM_COLS = 2 * BN;              // two accumulators
 
 struct GemmMaps {
     CUtensorMap a;
@@ -75,28 +75,41 @@ struct GemmMaps {
     CUtensorMap c[3];
 };
 
-__global__ void __launch_bounds__(GEMM_THREADS, 2)
-gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, DeviceCounters* dc) {
+struct TileCoord {
+    int w, m0, n0;
+};
+// Tile t of the launch: column tiles fastest, then row tiles, then the weight matrix, so that CTAs
+// working side by side share the A row panel in L2.
+__device__ __forceinline__ TileCoord tile_coord(int t, int mt, int nt) {
+    TileCoord c;
+    c.n0 = (t % nt) * BN;
+    const int r = t / nt;
+    c.m0 = (r % mt) * BM;
+    c.w = r / mt;
+    return c;
+}
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, int nW, DeviceCounters* dc) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_bar;
+    uint8_t* stage_out = smem + STAGES * STAGE_BYTES;
+    __shared__ uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int w = blockIdx.z;
-    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int nk = (K + BK - 1) / BK;
-    const CUtensorMap* mapB = &maps.b[w];
-    const CUtensorMap* mapC = &maps.c[w];
+    const int mt = (M + BM - 1) / BM, nt = (N + BN - 1) / BN;
+    const int ntiles = mt * nt * nW;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        mbar_init(&acc_bar, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
         fence_mbar_init();
     }
-    if (warp == 0) { tmem_alloc(&tmem_base_s, BN); tmem_relinquish(); }
+    if (warp == 1) { tmem_alloc(&tmem_base_s, TMEM_COLS); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -104,22 +117,25 @@ gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, Dev
     volatile int* abortp = &abort_flag;
 
     if (warp == 0 && lane == 0) {
-        // ---- TMA producer
-        int issued = 0;
-        for (int kt = 0; kt < nk; ++kt) {
-            const int s = kt % STAGES;
-            if (kt >= STAGES && !mbar_wait(&empty_bar[s], ((kt / STAGES) - 1) & 1, abortp)) break;
-            uint8_t* sA = smem + s * STAGE_BYTES;
-            uint8_t* sB = sA + A_BYTES;
-            mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
-            tma_load_2d(sA, &maps.a, &full_bar[s], kt * BK, m0);
+        // ---- TMA producer: k-steps of all this CTA's tiles, numbered g = 0, 1, ... through the ring
+        int g = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+            const TileCoord c = tile_coord(t, mt, nt);
+            for (int kt = 0; kt < nk; ++kt, ++g) {
+                const int s = g % STAGES;
+                if (g >= STAGES && !mbar_wait(&empty_bar[s], ((g / STAGES) - 1) & 1, abortp)) { ok = false; break; }
+                uint8_t* sA = smem + s * STAGE_BYTES;
+                uint8_t* sB = sA + A_BYTES;
+                mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
+                tma_load_2d(sA, &maps.a, &full_bar[s], kt * BK, c.m0);
 #pragma unroll
-            for (int u = 0; u < NSUB; ++u) tma_load_2d(sB + u * B_SUB_BYTES, mapB, &full_bar[s], n0 + 64 * u, kt * BK);
-            ++issued;
+                for (int u = 0; u < NSUB; ++u)
+                    tma_load_2d(sB + u * B_SUB_BYTES, &maps.b[c.w], &full_bar[s], c.n0 + 64 * u, kt * BK);
+            }
         }
         if (*abortp) {  // let copies already in flight land before the CTA goes away
-            for (int kt = max(0, issued - STAGES); kt < issued; ++kt)
-                mbar_wait_drain(&full_bar[kt % STAGES], (kt / STAGES) & 1);
+            for (int k = max(0, g - STAGES); k < g; ++k) mbar_wait_drain(&full_bar[k % STAGES], (k / STAGES) & 1);
         }
     } else if (warp == 1 && lane == 0) {
         // ---- MMA issuer
@@ -127,81 +143,111 @@ gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, Dev
         // descriptor low words of stage 0; a stage or k-step is a constant added to them (sm100.cuh)
         const uint32_t a_lo0 = umma_desc_lo_kmajor(smem_u32(smem));
         const uint32_t b_lo0 = umma_desc_lo_mnmajor(smem_u32(smem + A_BYTES), B_SUB_BYTES);
+        unsigned long long macs = 0;
+        int g = 0, i = 0;
         bool ok = true;
-        for (int kt = 0; kt < nk && ok; ++kt) {
-            const int s = kt % STAGES;
-            ok = mbar_wait(&full_bar[s], (kt / STAGES) & 1, abortp);
+        for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++i) {
+            const int buf = i & 1;
+            if (i >= 2) ok = mbar_wait(&acc_empty[buf], ((i >> 1) - 1) & 1, abortp);   // epilogue drained it
             if (!ok) break;
             tc_fence_after();
-            const uint32_t a_lo = a_lo0 + s * (STAGE_BYTES >> 4), b_lo = b_lo0 + s * (STAGE_BYTES >> 4);
-            if (kt == 0) {
+            const uint32_t acc = tmem + buf * BN;
+            for (int kt = 0; kt < nk; ++kt, ++g) {
+                const int s = g % STAGES;
+                ok = mbar_wait(&full_bar[s], (g / STAGES) & 1, abortp);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_lo = a_lo0 + s * (STAGE_BYTES >> 4), b_lo = b_lo0 + s * (STAGE_BYTES >> 4);
+                if (kt == 0) {
 #pragma unroll
-                for (int k = 0; k < BK / 16; ++k)
-                    umma_ss(tmem, umma_desc_join(a_lo + k * (32 >> 4), UMMA_DESC_HI_SW128),
-                            umma_desc_join(b_lo + k * (2048 >> 4), UMMA_DESC_HI_SW128), idesc, k != 0);
-            } else {
+                    for (int k = 0; k < BK / 16; ++k)
+                        umma_ss(acc, umma_desc_join(a_lo + k * (32 >> 4), UMMA_DESC_HI_SW128),
+                                umma_desc_join(b_lo + k * (2048 >> 4), UMMA_DESC_HI_SW128), idesc, k != 0);
+                } else {
 #pragma unroll
-                for (int k = 0; k < BK / 16; ++k)
-                    umma_ss(tmem, umma_desc_join(a_lo + k * (32 >> 4), UMMA_DESC_HI_SW128),
-                            umma_desc_join(b_lo + k * (2048 >> 4), UMMA_DESC_HI_SW128), idesc, 1);
+                    for (int k = 0; k < BK / 16; ++k)
+                        umma_ss(acc, umma_desc_join(a_lo + k * (32 >> 4), UMMA_DESC_HI_SW128),
+                                umma_desc_join(b_lo + k * (2048 >> 4), UMMA_DESC_HI_SW128), idesc, 1);
+                }
+                umma_commit(&empty_bar[s]);
             }
-            umma_commit(&empty_bar[s]);
+            if (!ok) break;
+            umma_commit(&acc_full[buf]);
+            const TileCoord c = tile_coord(t, mt, nt);
+            macs += (unsigned long long)min(BM, M - c.m0) * min(BN, N - c.n0) * K;
         }
-        if (ok) {
-            umma_commit(&acc_bar);
-            const unsigned long long vm = min(BM, M - m0), vn = min(BN, N - n0);
-            atomicAdd(&dc->proj_macs, vm * vn * (unsigned long long)K);
-        }
-    } else if (warp >= 2) {
+        if (macs) atomicAdd(&dc->proj_macs, macs);
+    }
+    else if (warp >= 2) {
         // ---- epilogue: 4 warps, warp q owns TMEM lanes 32q .. 32q+31 = output rows
         const int q = warp & 3;
         const int row = q * 32 + lane;
-        const bool ready = mbar_wait(&acc_bar, 0, abortp);
-        if (named_bar_all(ready, 1, 128)) {  // uniform across the four epilogue warps
-            tc_fence_after();
-            uint8_t* stage = smem;  // the ring is drained: every load landed and every MMA completed
+        int i = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++i) {
+            const int buf = i & 1;
+            if (ok) ok = mbar_wait(&acc_full[buf], (i >> 1) & 1, abortp);
+            const TileCoord c = tile_coord(t, mt, nt);
+            bool live = true;
+#pragma unroll 1
+            for (int hh = 0; hh < BN / OUT_COLS; ++hh) {
+                // uniform across the four warps; also orders the previous output store (warp 2 lane 0 waited
+                // for it to have read the staging buffer) before the writes below
+                if (!named_bar_all(ok, 1, 128)) { live = false; break; }
+                tc_fence_after();
 #pragma unroll
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld32(tmem + (static_cast<uint32_t>(q * 32) << 16) + c0, r);
-                tc_wait_ld();
-                uint8_t* sub = stage + (c0 / 64) * (BM * 128);
+                for (int c0 = 0; c0 < OUT_COLS; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem + (static_cast<uint32_t>(q * 32) << 16) + buf * BN + hh * OUT_COLS + c0, r);
+                    tc_wait_ld();
+                    uint8_t* sub = stage_out + (c0 / 64) * 16384;
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {  // four 16-byte chunks of 8 bf16
-                    uint4 v;
-                    v.x = pack_bf16x2(__uint_as_float(r[g * 8 + 0]), __uint_as_float(r[g * 8 + 1]));
-                    v.y = pack_bf16x2(__uint_as_float(r[g * 8 + 2]), __uint_as_float(r[g * 8 + 3]));
-                    v.z = pack_bf16x2(__uint_as_float(r[g * 8 + 4]), __uint_as_float(r[g * 8 + 5]));
-                    v.w = pack_bf16x2(__uint_as_float(r[g * 8 + 6]), __uint_as_float(r[g * 8 + 7]));
-                    *reinterpret_cast<uint4*>(sub + swz128_offset(row, (c0 % 64) / 8 + g)) = v;
+                    for (int g = 0; g < 4; ++g) {  // four 16-byte chunks of 8 bf16
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(r[g * 8 + 0]), __uint_as_float(r[g * 8 + 1]));
+                        v.y = pack_bf16x2(__uint_as_float(r[g * 8 + 2]), __uint_as_float(r[g * 8 + 3]));
+                        v.z = pack_bf16x2(__uint_as_float(r[g * 8 + 4]), __uint_as_float(r[g * 8 + 5]));
+                        v.w = pack_bf16x2(__uint_as_float(r[g * 8 + 6]), __uint_as_float(r[g * 8 + 7]));
+                        *reinterpret_cast<uint4*>(sub + swz128_offset(row, (c0 % 64) / 8 + g)) = v;
+                    }
+                }
+                if (hh == BN / OUT_COLS - 1) {
+                    tc_fence_before();
+                    mbar_arrive(&acc_empty[buf]);      // the accumulator may be overwritten by tile i + 2
+                }
+                fence_async_smem();
+                named_bar_sync(2, 128);
+                if (warp == 2 && lane == 0) {
+                    for (int u = 0; u < OUT_COLS / 64; ++u) {
+                        const int col = c.n0 + hh * OUT_COLS + 64 * u;
+                        if (col < N) tma_store_2d(&maps.c[c.w], stage_out + u * 16384, col, c.m0);
+                    }
+                    tma_store_commit();
+                    tma_store_wait_read();             // the staging buffer may be rewritten
                 }
             }
-            fence_async_smem();
-            named_bar_sync(1, 128);
-            if (warp == 2 && lane == 0) {
-#pragma unroll
-                for (int u = 0; u < NSUB; ++u)
-                    if (n0 + 64 * u < N) tma_store_2d(mapC, stage + u * (BM * 128), n0 + 64 * u, m0);
-                tma_store_commit();
-                tma_store_wait_all();
-            }
+            if (!live) { ok = false; break; }
         }
+        if (warp == 2 && lane == 0) tma_store_wait_all();
     }
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && abort_flag) atomicExch(&dc->status, (int)PSA_ERR_TIMEOUT);
-    if (warp == 0) tmem_dealloc(tmem, BN);
+    if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
 }  // namespace
 
 int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int nW, int M, int K, int N,
                  DeviceCounters* dc, cudaStream_t stream) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static int sm_count = 0;
+    if (!sm_count) {
         cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
-        if (e != cudaSuccess) { set_cuda_error(e, "cudaFuncSetAttribute(gemm)"); return PSA_ERR_CUDA; }
-        attr_set = true;
+        int dev = 0, sms = 0;
+        if (e == cudaSuccess) e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess || sms <= 0) { set_cuda_error(e, "gemm set-up"); return PSA_ERR_CUDA; }
+        sm_count = sms;
     }
     GemmMaps maps;
     if (!make_tensor_map_bf16(&maps.a, A, M, K, (uint64_t)K * 2, BM, BK)) return PSA_ERR_CUDA;
@@ -210,8 +256,9 @@ int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int n
         if (!make_tensor_map_bf16(&maps.b[w], Bw[src], K, N, (uint64_t)N * 2, BK, 64)) return PSA_ERR_CUDA;
         if (!make_tensor_map_bf16(&maps.c[w], C[src], M, N, (uint64_t)N * 2, BM, 64)) return PSA_ERR_CUDA;
     }
-    dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM, nW);
-    gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(maps, M, N, K, dc);
+    const int ntiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN) * nW;
+    const int grid = ntiles < sm_count ? ntiles : sm_count;
+    gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(maps, M, N, K, nW, dc);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "gemm_bf16_kernel launch"); return PSA_ERR_CUDA; }
     return PSA_OK;
