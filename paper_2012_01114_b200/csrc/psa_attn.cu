@@ -63,7 +63,10 @@ struct AttnCfg {
     static constexpr int KSTAGES = D == 128 ? 2 : 4;
     static constexpr int VSTAGES = D == 128 ? 2 : 4;
     static constexpr int SMEM = (2 + KSTAGES + VSTAGES) * TILE_BYTES + 1024;
-    static constexpr int TMEM_S = 0, TMEM_O = 256;
+    // With d = 64 the 512 TMEM columns have room for P outside S (S0 S1 | P0 P1 | O0 O1): S_{j+1} can then be
+    // computed while the softmax of block j is still running.  With d = 128 P overlays S.
+    static constexpr bool SEP_P = D == 64;
+    static constexpr int TMEM_S = 0, TMEM_P = 256, TMEM_O = SEP_P ? 384 : 256;
     // of every 4 consecutive elements, this many take the polynomial exp2 (FMA pipe) instead of MUFU
     static constexpr int POLY_OF_4 = PSA_POLY_OF_4;
 };
@@ -75,7 +78,7 @@ struct AttnMaps {
 struct AttnBars {
     uint64_t q_full[2];
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[2], p_ready[2], o_done[2];
+    uint64_t s_full[2], p_ready[2], o_done[2], s_free[2];
 };
 
 __device__ __forceinline__ float ex2_mufu(float x) {
@@ -195,6 +198,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bars.q_full[t], 1);
             mbar_init(&bars.s_full[t], 1);
+            mbar_init(&bars.s_free[t], 32 * SOFTMAX_WARPS_PER_TILE);
             mbar_init(&bars.p_ready[t], 32 * SOFTMAX_WARPS_PER_TILE);
             mbar_init(&bars.o_done[t], 1);
         }
@@ -248,6 +252,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
             const uint32_t idescO = umma_idesc_bf16(128, D, UMMA_K_MAJOR, UMMA_MN_MAJOR);
             unsigned long long qk_blocks = 0, pv_blocks = 0;
             bool ok = true;
+            constexpr bool SEP = Cfg::SEP_P && !SYM;
             // Descriptor low words of the operand bases; per MMA only a constant is added (sm100.cuh).
             const uint32_t q_lo0 = umma_desc_lo_kmajor(smem_u32(sQ)), q_lo1 = umma_desc_lo_kmajor(smem_u32(sQ + Cfg::TILE_BYTES));
             const uint32_t k_lo = umma_desc_lo_kmajor(smem_u32(sK));
@@ -277,6 +282,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                 tc_fence_after();
                 const uint32_t v = v_lo + sv * (Cfg::TILE_BYTES >> 4);
                 const uint32_t dO = tO0 + t * D, aP = tS0 + t * 128;
+                (void)aP;
                 if (j == 0) {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
@@ -309,11 +315,66 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                     umma_commit(&bars.k_empty[0]);
                 }
             }
-            for (int j = 0; j < maxkv && ok; ++j)
-                for (int t = 0; t < work.ntiles && ok; ++t) {
-                    const int nkv_t = t == 0 ? nkv0 : nkv1;
-                    if (j < nkv_t) ok = issue_step(t, j, !SYM && j + 1 < nkv_t);
+            if (!SEP) {
+                for (int j = 0; j < maxkv && ok; ++j)
+                    for (int t = 0; t < work.ntiles && ok; ++t) {
+                        const int nkv_t = t == 0 ? nkv0 : nkv1;
+                        if (j < nkv_t) ok = issue_step(t, j, !SYM && j + 1 < nkv_t);
+                    }
+            } else {
+                // Separate P: S_t(j+1) needs only that the softmax warps have taken S_t(j) out of TMEM
+                // (s_free) and PV_t(j) only P_t(j) (p_ready); the two tiles' events arrive in no fixed
+                // order, so the issuer polls them without blocking and issues whatever has become possible.
+                int nS[2] = {1, 1}, nPV[2] = {0, 0};
+                const int nkv[2] = {nkv0, nkv1};
+                const uint64_t t_start = globaltimer_ns();
+                uint32_t idle = 0;
+                while (ok && (nPV[0] < nkv0 || nPV[1] < nkv1)) {
+                    bool progressed = false;
+                    for (int t = 0; t < work.ntiles && ok; ++t) {
+                        const int o = t ^ 1;
+                        int j = nS[t];
+                        // (the operand tile is tested, not waited for: its load may itself depend on an MMA
+                        // of the other tile that this very thread has yet to issue)
+                        if (j < nkv[t] && mbar_test(&bars.s_free[t], (j - 1) & 1) &&
+                            mbar_test(&bars.k_full[j % Cfg::KSTAGES], (j / Cfg::KSTAGES) & 1)) {
+                            const int sk = j % Cfg::KSTAGES;
+                            tc_fence_after();
+                            mma_S(t, j);
+                            umma_commit(&bars.s_full[t]);
+                            ++nS[t];
+                            if (o >= work.ntiles || j >= nkv[o] || nS[o] > j) umma_commit(&bars.k_empty[sk]);
+                            progressed = true;
+                        }
+                        j = nPV[t];
+                        if (j < nkv[t] && mbar_test(&bars.p_ready[t], j & 1) &&
+                            mbar_test(&bars.v_full[j % Cfg::VSTAGES], (j / Cfg::VSTAGES) & 1)) {
+                            const int sv = j % Cfg::VSTAGES;
+                            tc_fence_after();
+                            const uint32_t v = v_lo + sv * (Cfg::TILE_BYTES >> 4);
+                            const uint32_t dO = tO0 + t * D, aP = tmem + Cfg::TMEM_P + t * 64;
+                            if (j == 0) {
+#pragma unroll
+                                for (int kk = 0; kk < 8; ++kk)
+                                    umma_ts(dO, aP + kk * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, kk != 0);
+                            } else {
+#pragma unroll
+                                for (int kk = 0; kk < 8; ++kk)
+                                    umma_ts(dO, aP + kk * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, 1);
+                            }
+                            ++pv_blocks;
+                            umma_commit(&bars.o_done[t]);
+                            ++nPV[t];
+                            if (o >= work.ntiles || j >= nkv[o] || nPV[o] > j) umma_commit(&bars.v_empty[sv]);
+                            progressed = true;
+                        }
+                    }
+                    if (!progressed && (++idle & 255u) == 0u) {
+                        if (*abortp) ok = false;
+                        else if (globaltimer_ns() - t_start > 4 * PSA_WAIT_LIMIT_NS) { *abortp = 1; ok = false; }
+                    }
                 }
+            }
             const unsigned long long block_macs = (unsigned long long)TILE * TILE * D;
             if (qk_blocks) atomicAdd(&dc->qk_macs, qk_blocks * block_macs);
             if (pv_blocks) {
@@ -331,12 +392,14 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
         const int t = sw / SOFTMAX_WARPS_PER_TILE;              // row tile of this warp
         const int part = (sw % SOFTMAX_WARPS_PER_TILE) >> 2;    // which share of the row's columns
         const int nkv = t == 0 ? nkv0 : nkv1;
+        constexpr bool SEP = Cfg::SEP_P && !SYM;
         if (t < work.ntiles) {
             const int q = warp & 3;                             // TMEM lane quarter this warp may access
             const int r = q * 32 + lane;                        // row inside the tile = TMEM lane
             const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
             const uint32_t tS = tmem + Cfg::TMEM_S + t * 128 + lane_off;
             const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off + part * OPT;
+            const uint32_t tP = tmem + Cfg::TMEM_P + t * 64 + lane_off;     // separate-P layout only
             const int It = work.tile0 + t;
             const int pair_bar = 1 + t * 4 + q;                 // named barrier of the warps sharing rows
             const int tile_bar = 9 + t;                         // named barrier of all softmax warps of the tile
@@ -345,9 +408,13 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
             float m_run = -INFINITY, l_run = 0.f;
             bool ok = true;
             for (int j = 0; j < nkv; ++j) {
-                // block 0 waits for the first S; later blocks for the commit that follows PV_{j-1} and S_j
-                if (j == 0) { if (!SYM) ok = mbar_wait(&bars.s_full[t], 0, abortp); }
-                else ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);
+                if (SEP) {
+                    ok = mbar_wait(&bars.s_full[t], j & 1, abortp);    // every S_j has its own commit
+                } else {
+                    // block 0 waits for the first S; later blocks for the commit that follows PV_{j-1} and S_j
+                    if (j == 0) { if (!SYM) ok = mbar_wait(&bars.s_full[t], 0, abortp); }
+                    else ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);
+                }
                 ok = __all_sync(0xffffffffu, ok);
                 if (TPR == 1 && !ok) break;
                 const bool diag = (scheme == PSA_MASKED) && (j == It);
@@ -400,16 +467,30 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                     for (int c = 0; c < NCH; ++c) load32(c, sreg[c]);
                     if (!SYM) tc_wait_ld();
                 }
+                if (SEP) {
+                    // S_j is in registers: the issuer may overwrite it with S_{j+1} while the exponentials run
+                    tc_fence_before();
+                    mbar_arrive(&bars.s_free[t]);
+                    // P and O are still in use by PV_{j-1} until its commit.  A wait given up here is not
+                    // acted on before the next pair barrier, so that the two threads of a row stay together.
+                    if (j > 0) {
+                        ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);
+                        ok = __all_sync(0xffffffffu, ok);
+                        tc_fence_after();
+                    }
+                }
+                if (ok) {
 #pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    uint32_t pk[16];
-                    const int kc = col_base + 32 * c;            // first key column of the chunk
-                    rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(sreg[c], sl2, -m_run, kc, r, pk)
-                                   : exp_chunk32<Cfg::POLY_OF_4, false>(sreg[c], sl2, -m_run, kc, r, pk);
-                    tmem_st16(tS + (kc >> 6) * 64 + ((kc & 63) >> 1), pk);
+                    for (int c = 0; c < NCH; ++c) {
+                        uint32_t pk[16];
+                        const int kc = col_base + 32 * c;            // first key column of the chunk
+                        rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(sreg[c], sl2, -m_run, kc, r, pk)
+                                       : exp_chunk32<Cfg::POLY_OF_4, false>(sreg[c], sl2, -m_run, kc, r, pk);
+                        tmem_st16(SEP ? tP + (kc >> 1) : tS + (kc >> 6) * 64 + ((kc & 63) >> 1), pk);
+                    }
                 }
                 l_run = fmaf(l_run, alpha, rowsum);
-                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8
+                if (ok && j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8
 #pragma unroll
                     for (int c = 0; c < OPT / 32; ++c) {
                         uint32_t v[32];
