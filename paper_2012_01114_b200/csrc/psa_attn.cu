@@ -40,6 +40,9 @@ namespace psa {
 
 namespace {
 
+#ifndef PSA_SOFTMAX_SLEEP_NS
+#define PSA_SOFTMAX_SLEEP_NS 0
+#endif
 #ifndef PSA_RELOAD_S
 #define PSA_RELOAD_S 1
 #endif
@@ -409,11 +412,11 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
             bool ok = true;
             for (int j = 0; j < nkv; ++j) {
                 if (SEP) {
-                    ok = mbar_wait(&bars.s_full[t], j & 1, abortp);    // every S_j has its own commit
+                    ok = mbar_wait<PSA_SOFTMAX_SLEEP_NS>(&bars.s_full[t], j & 1, abortp);    // every S_j has its own commit
                 } else {
                     // block 0 waits for the first S; later blocks for the commit that follows PV_{j-1} and S_j
-                    if (j == 0) { if (!SYM) ok = mbar_wait(&bars.s_full[t], 0, abortp); }
-                    else ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);
+                    if (j == 0) { if (!SYM) ok = mbar_wait<PSA_SOFTMAX_SLEEP_NS>(&bars.s_full[t], 0, abortp); }
+                    else ok = mbar_wait<PSA_SOFTMAX_SLEEP_NS>(&bars.o_done[t], (j - 1) & 1, abortp);
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (TPR == 1 && !ok) break;

@@ -83,11 +83,13 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait for the phase with the given parity to complete.  `abort_flag` lives in shared
 // memory; any thread that gives up sets it and every other waiter leaves at its next poll.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
     uint32_t it = 0;
     while (!mbar_try_wait(bar, parity)) {
+        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);   // waiters that are many (softmax warps) yield their issue slots
         if ((++it & 63u) == 0u) {
             if (*abort_flag) return false;
             if (globaltimer_ns() - t0 > PSA_WAIT_LIMIT_NS) {
