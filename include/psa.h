@@ -64,7 +64,7 @@ typedef enum {
  *   useful_*        the paper's element-level counts for the scheme (Sec. 3.2, 4.2, 5.2):
  *                   FULL d*n^2 each; MASKED d*n(n+1)/2 each; SYMMETRIC d*n(n+1)/2 and d*n^2
  * The bf16 path issues whole 128x128 blocks of the weight matrix, so issued >= useful there (a
- * block on the diagonal is issued in full); the fp32 path skips element by element, issued = useful.
+ * block on the diagonal, or a ragged last block, is issued in full); the fp32 path skips element by element, issued = useful.
  */
 typedef struct {
     uint64_t proj_macs, qk_macs, pv_macs, exps, useful_qk_macs, useful_pv_macs;
@@ -74,7 +74,8 @@ typedef struct {
  * Projections + attention, bf16 in / bf16 out, fp32 accumulation (paper Sec. 3.1 then Eq. 1-3).
  *   X, Wq, Wk, Wv, out   device, bf16, layouts above.
  *   PSA_SYMMETRIC: q = k = v = X*Wq (paper Sec. 4.1); Wk and Wv must be NULL or equal to Wq.
- * Supported: d_k in {64, 128}; n a multiple of 128; d_model and heads*d_k multiples of 64.
+ * Supported: d_k in {64, 128}; any n >= 1 (a last block of fewer than 128 vectors is zero-filled and its
+ * keys carry no weight); d_model and heads*d_k multiples of 64.
  * Needs a workspace of psa_workspace_bytes(...) (grown on demand, see psa_set_workspace).
  */
 int psa_attention(const void* X, const void* Wq, const void* Wk, const void* Wv, int batch, int heads, int n,

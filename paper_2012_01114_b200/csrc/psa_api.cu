@@ -44,7 +44,6 @@ int check_shape(int batch, int heads, int n, int d_model, int d_k, int scheme, i
     if ((long long)batch * n > 0x7fffffffLL || (long long)heads * d_k > 0x7fffffffLL) return PSA_ERR_SHAPE;
     if (dtype == PSA_BF16) {
         if (d_k != 64 && d_k != 128) return PSA_ERR_UNSUPPORTED;
-        if (n % TILE != 0) return PSA_ERR_UNSUPPORTED;
         if (with_proj && (d_model % 64 != 0)) return PSA_ERR_UNSUPPORTED;
     } else {
         if (n > 1024 || d_k > 128) return PSA_ERR_UNSUPPORTED;

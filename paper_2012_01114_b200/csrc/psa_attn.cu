@@ -170,7 +170,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
     const CtaWork work = cta_work(blockIdx.x, n, scheme == PSA_MASKED, nbh, global_lpt);
     const int bh = bh0 + work.bh;
     const int b = bh / H, h = bh - b * H;
-    const int row0 = b * n, col0 = h * D;
+    const int col0 = h * D;
     const int nkv0 = kv_tiles(work.tile0, T, scheme);
     const int nkv1 = work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0;
     const int maxkv = max(nkv0, nkv1);
@@ -180,21 +180,21 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
     auto load_q = [&](int t) {
         mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
         for (int u = 0; u < Cfg::SUB; ++u)
-            tma_load_2d(sQ + t * Cfg::TILE_BYTES + u * 16384, &maps.q, &bars.q_full[t], col0 + 64 * u,
-                        row0 + (work.tile0 + t) * TILE);
+            tma_load_3d(sQ + t * Cfg::TILE_BYTES + u * 16384, &maps.q, &bars.q_full[t], col0 + 64 * u,
+                        (work.tile0 + t) * TILE, b);
     };
     auto load_k = [&](int j) {
         if (SYM) return;
         const int s = j % Cfg::KSTAGES;
         mbar_arrive_expect_tx(&bars.k_full[s], Cfg::TILE_BYTES);
         for (int u = 0; u < Cfg::SUB; ++u)
-            tma_load_2d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], col0 + 64 * u, row0 + j * TILE);
+            tma_load_3d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], col0 + 64 * u, j * TILE, b);
     };
     auto load_v = [&](int j) {
         const int s = j % Cfg::VSTAGES;
         mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
         for (int u = 0; u < Cfg::SUB; ++u)
-            tma_load_2d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], col0 + 64 * u, row0 + j * TILE);
+            tma_load_3d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], col0 + 64 * u, j * TILE, b);
     };
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -407,7 +407,8 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
             const int pair_bar = 1 + t * 4 + q;                 // named barrier of the warps sharing rows
             const int tile_bar = 9 + t;                         // named barrier of all softmax warps of the tile
             const int col_base = part * CPT;
-            const float* srow = SYM ? Sg + ((size_t)work.bh * n + (size_t)It * TILE + r) * n + col_base : nullptr;
+            const size_t npad = (size_t)T * TILE;                 // S scratch is [heads, npad, npad]
+            const float* srow = SYM ? Sg + ((size_t)work.bh * npad + (size_t)It * TILE + r) * npad + col_base : nullptr;
             float m_run = -INFINITY, l_run = 0.f;
             bool ok = true;
             for (int j = 0; j < nkv; ++j) {
@@ -420,7 +421,12 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (TPR == 1 && !ok) break;
-                const bool diag = (scheme == PSA_MASKED) && (j == It);
+                // Element predicate: on the diagonal block of the masked scheme keys beyond the row's own index,
+                // and on a ragged last block keys beyond the sequence, carry no weight.  `cb` = last kept column.
+                const int nvalid = min(TILE, n - j * TILE);
+                const bool on_diag = (scheme == PSA_MASKED) && (j == It);
+                const bool diag = on_diag || nvalid < TILE;
+                const int cb = min(on_diag ? r : TILE - 1, nvalid - 1);
                 float mx = -INFINITY;
                 // 32 raw scores of this thread's share of the row: chunk c = block columns col_base + 32c ..
                 auto load32 = [&](int c, uint32_t (&v)[32]) {
@@ -445,7 +451,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                     if (!SYM) tc_wait_ld();
 #pragma unroll
                     for (int c = 0; c < NCH; ++c)
-                        mx = diag ? max_chunk32<true>(sreg[c], col_base + 32 * c, r, mx)
+                        mx = diag ? max_chunk32<true>(sreg[c], col_base + 32 * c, cb, mx)
                                   : max_chunk32<false>(sreg[c], col_base + 32 * c, r, mx);
                 }
                 if (TPR == 2) {
@@ -487,7 +493,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                     for (int c = 0; c < NCH; ++c) {
                         uint32_t pk[16];
                         const int kc = col_base + 32 * c;            // first key column of the chunk
-                        rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(sreg[c], sl2, -m_run, kc, r, pk)
+                        rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(sreg[c], sl2, -m_run, kc, cb, pk)
                                        : exp_chunk32<Cfg::POLY_OF_4, false>(sreg[c], sl2, -m_run, kc, r, pk);
                         tmem_st16(SEP ? tP + (kc >> 1) : tS + (kc >> 6) * 64 + ((kc & 63) >> 1), pk);
                     }
@@ -536,7 +542,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
                 named_bar_sync(tile_bar, 32 * SOFTMAX_WARPS_PER_TILE);
                 if (sw == t * SOFTMAX_WARPS_PER_TILE && lane == 0) {
                     for (int u = 0; u < Cfg::SUB; ++u)
-                        tma_store_2d(&maps.o, stage + u * 16384, col0 + 64 * u, row0 + It * TILE);
+                        tma_store_3d(&maps.o, stage + u * 16384, col0 + 64 * u, It * TILE, b);
                     tma_store_commit();
                     tma_store_wait_read();   // smem may be released; the writes complete on their own
                 }
@@ -574,7 +580,8 @@ sym_scores_kernel(const __grid_constant__ CUtensorMap mapX, float* __restrict__ 
     int I, J;
     sym_pair(blockIdx.x - hl * np, &I, &J);
     const int bh = bh0 + hl, b = bh / H, h = bh - b * H;
-    const int row0 = b * n, col0 = h * D;
+    const int col0 = h * D;
+    const size_t npad = (size_t)T * TILE;            // the scratch is padded to whole tiles
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -592,8 +599,8 @@ sym_scores_kernel(const __grid_constant__ CUtensorMap mapX, float* __restrict__ 
     if (threadIdx.x == 0) {
         mbar_arrive_expect_tx(&full_bar, 2 * TILE_BYTES);
         for (int u = 0; u < SUB; ++u) {
-            tma_load_2d(sA + u * 16384, &mapX, &full_bar, col0 + 64 * u, row0 + I * TILE);
-            tma_load_2d(sB + u * 16384, &mapX, &full_bar, col0 + 64 * u, row0 + J * TILE);
+            tma_load_3d(sA + u * 16384, &mapX, &full_bar, col0 + 64 * u, I * TILE, b);
+            tma_load_3d(sB + u * 16384, &mapX, &full_bar, col0 + 64 * u, J * TILE, b);
         }
         if (mbar_wait(&full_bar, 0, abortp)) {
             tc_fence_after();
@@ -614,7 +621,7 @@ sym_scores_kernel(const __grid_constant__ CUtensorMap mapX, float* __restrict__ 
     const bool ready = mbar_wait(&acc_bar, 0, abortp);
     if (__syncthreads_and(ready)) {
         tc_fence_after();
-        float* Sh = Sg + (size_t)hl * n * n;
+        float* Sh = Sg + (size_t)hl * npad * npad;
         const int r = warp * 32 + lane;
 #pragma unroll 1
         for (int c0 = 0; c0 < 128; c0 += 32) {
@@ -626,12 +633,12 @@ sym_scores_kernel(const __grid_constant__ CUtensorMap mapX, float* __restrict__ 
                 const float s = __uint_as_float(v[i]) * scale;
                 tr[warp][lane][i] = s;
                 if (I != J)  // mirror block: element (J*128 + c0 + i, I*128 + r); lanes run along a row
-                    Sh[((size_t)J * TILE + c0 + i) * n + (size_t)I * TILE + r] = s;
+                    Sh[((size_t)J * TILE + c0 + i) * npad + (size_t)I * TILE + r] = s;
             }
             __syncwarp();
 #pragma unroll
             for (int rr = 0; rr < 32; ++rr)  // direct block, lanes run along a row
-                Sh[((size_t)I * TILE + warp * 32 + rr) * n + (size_t)J * TILE + c0 + lane] = tr[warp][rr][lane];
+                Sh[((size_t)I * TILE + warp * 32 + rr) * npad + (size_t)J * TILE + c0 + lane] = tr[warp][rr][lane];
             __syncwarp();
         }
     }
@@ -644,7 +651,8 @@ sym_scores_kernel(const __grid_constant__ CUtensorMap mapX, float* __restrict__ 
 constexpr size_t SYM_SCRATCH_CAP = size_t(2) << 30;  // bytes of score scratch per pass
 
 int sym_heads_per_pass(int B, int H, int n) {
-    const size_t per_head = (size_t)n * n * sizeof(float);
+    const size_t npad = (size_t)row_tiles(n) * TILE;
+    const size_t per_head = npad * npad * sizeof(float);
     size_t hp = SYM_SCRATCH_CAP / per_head;
     if (hp < 1) hp = 1;
     if (hp > (size_t)B * H) hp = (size_t)B * H;
@@ -666,12 +674,10 @@ int launch_attention(const void* Q, const void* K, const void* V, void* out, flo
         if (e != cudaSuccess) { set_cuda_error(e, "cudaFuncSetAttribute(attention)"); return PSA_ERR_CUDA; }
         attr_set = true;
     }
-    const uint64_t rows = (uint64_t)B * n, cols = (uint64_t)H * D, pitch = cols * 2;
+    const uint64_t cols = (uint64_t)H * D;
     AttnMaps maps;
-    if (!make_tensor_map_bf16(&maps.q, Q, rows, cols, pitch, 128, 64) ||
-        !make_tensor_map_bf16(&maps.k, K, rows, cols, pitch, 128, 64) ||
-        !make_tensor_map_bf16(&maps.v, V, rows, cols, pitch, 128, 64) ||
-        !make_tensor_map_bf16(&maps.o, out, rows, cols, pitch, 128, 64))
+    if (!make_tensor_map_bf16_3d(&maps.q, Q, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.k, K, B, n, cols, 128) ||
+        !make_tensor_map_bf16_3d(&maps.v, V, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.o, out, B, n, cols, 128))
         return PSA_ERR_CUDA;
     const int P = ctas_per_head(n);
     cudaError_t e;
@@ -700,7 +706,8 @@ int launch_attention(const void* Q, const void* K, const void* V, void* out, flo
 }  // namespace
 
 size_t bf16_symmetric_scratch_bytes(int B, int H, int n) {
-    return (size_t)sym_heads_per_pass(B, H, n) * n * n * sizeof(float);
+    const size_t npad = (size_t)row_tiles(n) * TILE;
+    return (size_t)sym_heads_per_pass(B, H, n) * npad * npad * sizeof(float);
 }
 
 int bf16_attention(const void* Q, const void* K, const void* V, void* out, float* S, size_t s_bytes, int B, int H,

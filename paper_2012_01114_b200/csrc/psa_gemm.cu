@@ -25,8 +25,8 @@ EncodeTiledFn g_encode = nullptr;
 std::once_flag g_encode_once;
 }  // namespace
 
-bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_bytes,
-                          uint32_t box_rows, uint32_t box_cols) {
+namespace {
+bool resolve_encode() {
     std::call_once(g_encode_once, [] {
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult q;
@@ -35,6 +35,13 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uin
             g_encode = reinterpret_cast<EncodeTiledFn>(fn);
     });
     if (!g_encode) { set_error_text("cuTensorMapEncodeTiled entry point not available"); return false; }
+    return true;
+}
+}  // namespace
+
+bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_bytes,
+                          uint32_t box_rows, uint32_t box_cols) {
+    if (!resolve_encode()) return false;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {pitch_bytes};
     cuuint32_t box[2] = {box_cols, box_rows};
@@ -45,6 +52,25 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uin
     if (r != CUDA_SUCCESS) {
         char msg[96];
         snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        set_error_text(msg);
+        return false;
+    }
+    return true;
+}
+
+bool make_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t batch, uint64_t n, uint64_t cols,
+                             uint32_t box_rows) {
+    if (!resolve_encode()) return false;
+    cuuint64_t dims[3] = {cols, n, batch};
+    cuuint64_t strides[2] = {cols * 2, n * cols * 2};
+    cuuint32_t box[3] = {64, box_rows, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char msg[96];
+        snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled (3-D) failed with CUresult %d", (int)r);
         set_error_text(msg);
         return false;
     }

@@ -27,7 +27,7 @@ struct CtaWork {
     int ntiles;    // 1 or 2 row tiles owned
 };
 
-PSA_HD int row_tiles(int n) { return n / TILE; }
+PSA_HD int row_tiles(int n) { return (n + TILE - 1) / TILE; }   // the last tile may be ragged
 PSA_HD int ctas_per_head(int n) { return (row_tiles(n) + TILES_PER_CTA - 1) / TILES_PER_CTA; }
 
 // CTA index -> work, for a launch over `nbh` (batch, head) units.

@@ -30,13 +30,19 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 @pytest.mark.parametrize("scheme", [oracle.FULL, oracle.SYMMETRIC, oracle.MASKED])
-@pytest.mark.parametrize("n,d", [(128, 64), (256, 128), (384, 64), (1024, 64), (1152, 128)])
+@pytest.mark.parametrize("n,d", [(128, 64), (256, 128), (384, 64), (1024, 64), (1152, 128), (1, 64), (100, 128), (129, 64),
+                                 (1000, 128)])
 def test_skip_count_bf16_matches_oracle_tile_census(lib, scheme, n, d):
+    # The kernels issue whole 128x128 blocks, also where the sequence ends inside a block: issued MACs are
+    # (number of blocks the oracle's enumeration keeps) x 128*128*d; for n % 128 == 0 that is the oracle's
+    # own issued figure.
     B, H = 3, 5
     c = binding.psa_skip_count(B, H, n, 0, d, scheme, binding.BF16)
     t = oracle.tile_counts(n, d, scheme, 128, 128)
-    assert c["qk_macs"] == B * H * t.issued_mac1
-    assert c["pv_macs"] == B * H * t.issued_mac3
+    assert c["qk_macs"] == B * H * t.tiles1 * 128 * 128 * d
+    assert c["pv_macs"] == B * H * t.tiles3 * 128 * 128 * d
+    if n % 128 == 0:
+        assert (c["qk_macs"], c["pv_macs"]) == (B * H * t.issued_mac1, B * H * t.issued_mac3)
     assert c["useful_qk_macs"] == B * H * t.useful_mac1
     assert c["useful_pv_macs"] == B * H * t.useful_mac3
     assert c["proj_macs"] == 0
@@ -67,7 +73,8 @@ def test_skip_fractions_track_the_papers_reductions(lib):
 def test_argument_errors_launch_nothing(lib):
     c = binding.Counts()
     assert lib.psa_skip_count(1, 1, 128, 0, 64, 7, binding.BF16, ctypes.byref(c)) == binding.ERR_SCHEME_ARGS
-    assert lib.psa_skip_count(1, 1, 100, 0, 64, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED
+    assert lib.psa_skip_count(1, 1, 100, 0, 64, 0, binding.BF16, ctypes.byref(c)) == binding.OK      # ragged n is fine
+    assert lib.psa_skip_count(1, 1, 128, 100, 64, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED  # d_model % 64
     assert lib.psa_skip_count(1, 1, 128, 0, 96, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED
     assert lib.psa_skip_count(1, 1, 2048, 0, 64, 0, binding.F32, ctypes.byref(c)) == binding.ERR_UNSUPPORTED
     assert lib.psa_skip_count(0, 1, 128, 0, 64, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_SHAPE
@@ -78,6 +85,6 @@ def test_argument_errors_launch_nothing(lib):
     assert lib.psa_attention_core(8, 16, 16, 1, 1, 128, 64, 0, binding.BF16, 16, None) == binding.ERR_ALIGN
     assert lib.psa_attention_core(16, 32, 16, 1, 1, 128, 64, 1, binding.BF16, 16, None) == binding.ERR_SCHEME_ARGS
     assert lib.psa_attention(16, 16, 32, 16, 1, 1, 128, 64, 64, 1, 16, None) == binding.ERR_SCHEME_ARGS
-    assert lib.psa_workspace_bytes(1, 1, 100, 0, 64, 0, binding.BF16, 0) == 0
+    assert lib.psa_workspace_bytes(1, 1, 100, 0, 96, 0, binding.BF16, 0) == 0
     assert binding.psa_status_string(binding.ERR_TIMEOUT).startswith("a bounded")
     assert binding.psa_workspace_bytes(8, 12, 1024, 768, 64, oracle.MASKED, binding.BF16) >= 3 * 8 * 1024 * 768 * 2

@@ -23,8 +23,8 @@ def _check_census(B, H, n, D, d, scheme):
     st, got = binding.psa_last_issued()
     assert st == binding.OK
     t = oracle.tile_counts(n, d, scheme, 128, 128)
-    assert got["qk_macs"] == B * H * t.issued_mac1
-    assert got["pv_macs"] == B * H * t.issued_mac3
+    assert got["qk_macs"] == B * H * t.tiles1 * 128 * 128 * d       # whole blocks are issued, ragged or not
+    assert got["pv_macs"] == B * H * t.tiles3 * 128 * 128 * d
     assert got["useful_qk_macs"] == B * H * t.useful_mac1
     assert got["useful_pv_macs"] == B * H * t.useful_mac3
     nproj = 0 if D == 0 else (1 if scheme == oracle.SYMMETRIC else 3)
@@ -68,6 +68,27 @@ def test_layer_with_projections_matches_oracle(scheme, B, H, n, D, d):
     err = np.abs(_to_f64(out) - ref).max()
     assert err <= TOL_BF16, err
     _check_census(B, H, n, D, d, scheme)
+
+
+@pytest.mark.parametrize("scheme", [oracle.FULL, oracle.MASKED, oracle.SYMMETRIC])
+@pytest.mark.parametrize("B,H,n,d", [(2, 2, 1, 64), (1, 3, 100, 128), (2, 1, 129, 64), (1, 2, 200, 128), (1, 2, 333, 64),
+                                     (2, 2, 1000, 128)])
+def test_ragged_sequence_lengths(scheme, B, H, n, d):
+    # n not a multiple of the 128-row block: the last block is zero-filled by TMA and its keys carry no weight
+    err = _core_case(B, H, n, d, scheme, seed=7 * n + d)
+    assert err <= TOL_BF16, err
+    _check_census(B, H, n, 0, d, scheme)
+
+
+def test_ragged_layer_with_projections():
+    B, H, n, D, d = 2, 2, 300, 128, 64
+    Xv, Xb = inputs.tensor(17, 0, (B, n, D), 1.0, "bf16")
+    W = [inputs.tensor(17, 1 + i, (D, H * d), D ** -0.5, "bf16") for i in range(3)]
+    out = binding.psa_attention(_dev_bf16(Xb), _dev_bf16(W[0][1]), _dev_bf16(W[1][1]), _dev_bf16(W[2][1]), H,
+                                binding.MASKED)
+    ref, _ = oracle.attention_layer(Xv, W[0][0], W[1][0], W[2][0], H, oracle.MASKED)
+    assert np.abs(_to_f64(out) - ref).max() <= TOL_BF16
+    _check_census(B, H, n, D, d, oracle.MASKED)
 
 
 def test_config2_shape_reduced_batch():
