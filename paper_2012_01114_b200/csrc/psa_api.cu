@@ -280,7 +280,7 @@ int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme
     uint64_t qk_blocks = 0, pv_blocks = 0;
     const int P = ctas_per_head(n);
     for (int cta = 0; cta < P; ++cta) {  // every head has the same list
-        const CtaWork w = cta_work(cta, n, scheme == PSA_MASKED, 1, 0);
+        const CtaWork w = cta_work(cta, n, scheme == PSA_MASKED, 1, 1);
         for (int t = 0; t < w.ntiles; ++t) {
             const int kv = kv_tiles(w.tile0 + t, T, scheme);
             pv_blocks += kv;

@@ -152,7 +152,7 @@ __device__ __forceinline__ float max_chunk32(const uint32_t (&s)[32], int col0, 
 template <int D, bool SYM>
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
 attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg, int n, int H, int scheme, int bh0,
-            int nbh, int global_lpt, float sl2, DeviceCounters* dc) {
+            int nbh, int group, float sl2, DeviceCounters* dc) {
     using Cfg = AttnCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -167,7 +167,7 @@ attn_kernel(const __grid_constant__ AttnMaps maps, const float* __restrict__ Sg,
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int T = row_tiles(n);
-    const CtaWork work = cta_work(blockIdx.x, n, scheme == PSA_MASKED, nbh, global_lpt);
+    const CtaWork work = cta_work(blockIdx.x, n, scheme == PSA_MASKED, nbh, group);
     const int bh = bh0 + work.bh;
     const int b = bh / H, h = bh - b * H;
     const int col0 = h * D;
@@ -683,7 +683,7 @@ int launch_attention(const void* Q, const void* K, const void* V, void* out, flo
     cudaError_t e;
     if (scheme != PSA_SYMMETRIC) {
         attn_kernel<D, false><<<B * H * P, ATTN_THREADS, Cfg::SMEM, stream>>>(maps, nullptr, n, H, scheme, 0, B * H,
-                                                                             use_global_lpt(scheme, (long long)B * H, n, D),
+                                                                             lpt_group(scheme, B * H, n, D),
                                                                              scale * LOG2E, dc);
         e = cudaGetLastError();
         if (e != cudaSuccess) { set_cuda_error(e, "attn_kernel launch"); return PSA_ERR_CUDA; }
@@ -696,7 +696,7 @@ int launch_attention(const void* Q, const void* K, const void* V, void* out, flo
         sym_scores_kernel<D><<<heads * np, 128, 2 * Cfg::TILE_BYTES + 1024, stream>>>(maps.q, S, n, H, bh0, scale, dc);
         e = cudaGetLastError();
         if (e != cudaSuccess) { set_cuda_error(e, "sym_scores_kernel launch"); return PSA_ERR_CUDA; }
-        attn_kernel<D, true><<<heads * P, ATTN_THREADS, Cfg::SMEM, stream>>>(maps, S, n, H, PSA_SYMMETRIC, bh0, heads, 0, LOG2E, dc);
+        attn_kernel<D, true><<<heads * P, ATTN_THREADS, Cfg::SMEM, stream>>>(maps, S, n, H, PSA_SYMMETRIC, bh0, heads, 1, LOG2E, dc);
         e = cudaGetLastError();
         if (e != cudaSuccess) { set_cuda_error(e, "attn_kernel(symmetric) launch"); return PSA_ERR_CUDA; }
     }

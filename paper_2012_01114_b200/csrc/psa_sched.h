@@ -30,34 +30,40 @@ struct CtaWork {
 PSA_HD int row_tiles(int n) { return (n + TILE - 1) / TILE; }   // the last tile may be ragged
 PSA_HD int ctas_per_head(int n) { return (row_tiles(n) + TILES_PER_CTA - 1) / TILES_PER_CTA; }
 
-// CTA index -> work, for a launch over `nbh` (batch, head) units.
-//   head-major order (global_lpt = 0): heads are the slow index so that CTAs resident together read the
-//     same K and V (L2 reuse); inside a head the masked scheme hands out the heaviest row tiles first.
-//   global order (global_lpt = 1, masked scheme on problems whose K and V all fit in L2 anyway): all heads'
-//     heaviest row-tile pairs first, then the next heaviest, ... so that the hardware's in-order CTA
-//     dispatch amounts to longest-processing-time-first scheduling.
-// Both play the role of the paper's pairing of long rows with short ones (Sec. 5.2): balance.
-PSA_HD CtaWork cta_work(int cta, int n, int scheme_masked, int nbh, int global_lpt) {
+// CTA index -> work, for a launch over `nbh` (batch, head) units taken in groups of `group` heads.
+// Inside a group the order is: every head's heaviest pair of row tiles first, then every head's next
+// heaviest, ... so that the hardware's in-order CTA dispatch amounts to longest-processing-time-first
+// scheduling over the group (the role of the paper's pairing of long rows with short ones, Sec. 5.2:
+// balance).  Groups follow one another, which keeps the K and V that concurrently running CTAs read
+// to one group's worth (L2 reuse).  group = 1 is plain head-major order.
+PSA_HD CtaWork cta_work(int cta, int n, int scheme_masked, int nbh, int group) {
     const int P = ctas_per_head(n);
+    const int full_groups = nbh / group;
+    int g = cta / (group * P);
+    if (g > full_groups) g = full_groups;
+    const int off = cta - g * group * P;
+    const int size = g < full_groups ? group : nbh - full_groups * group;   // heads in this group
+    const int r = off / size;
     CtaWork w;
-    int r;
-    if (global_lpt) {
-        r = cta / nbh;
-        w.bh = cta - r * nbh;
-    } else {
-        w.bh = cta / P;
-        r = cta - w.bh * P;
-    }
+    w.bh = g * group + (off - r * size);
     const int p = scheme_masked ? (P - 1 - r) : r;
     w.tile0 = p * TILES_PER_CTA;
     const int left = row_tiles(n) - w.tile0;
     w.ntiles = left < TILES_PER_CTA ? left : TILES_PER_CTA;
     return w;
 }
-// Whether a masked launch uses the global order: K and V of every head together stay below this many bytes.
-constexpr long long GLOBAL_LPT_MAX_KV_BYTES = 48ll << 20;
-PSA_HD int use_global_lpt(int scheme, long long nbh, int n, int d) {
-    return scheme == PSA_MASKED && nbh * n * d * 2 * 2 <= GLOBAL_LPT_MAX_KV_BYTES;
+// Heads per group: as many as keep the group's K and V (bf16) within a fraction of L2; the schemes whose
+// CTAs all do the same work gain nothing from reordering and keep head-major order.
+#ifndef PSA_LPT_MB
+#define PSA_LPT_MB 64
+#endif
+PSA_HD int lpt_group(int scheme, int nbh, int n, int d) {
+    if (scheme != PSA_MASKED) return 1;
+    const long long per_head = (long long)n * d * 2 * 2;
+    long long g = ((long long)PSA_LPT_MB << 20) / per_head;
+    if (g < 1) g = 1;
+    if (g > nbh) g = nbh;
+    return (int)g;
 }
 
 // Number of key/value tiles row tile I visits in phases 1-3 of the fused kernel (FULL, MASKED) or
