@@ -1,0 +1,550 @@
+// Fused attention core of the bf16 path for the FULL and MASKED schemes: phases 1-3 of the paper
+// (Eq. 1-3) per (batch, head) and pair of 128-row query tiles, never materialising the n x n weight
+// matrix, as ONE persistent kernel: a CTA per SM walks the tile scheduler's work list.
+//
+//   phase 1  S = Q K^T            tcgen05 MMA, operands staged by TMA, accumulator in TMEM
+//   phase 2  softmax              two threads per query row (64 columns each) read S from TMEM, keep a
+//                                 running row maximum m and row sum l (the division of Eq. 2 is
+//                                 applied once to the output row), write P = exp2(..) as bf16 to TMEM
+//   phase 3  O += P V             tcgen05 MMA with P read from TMEM and V (row-major = MN-major) from
+//                                 shared memory, accumulator O in TMEM
+//
+// Which (row tile, column tile) blocks exist is decided by the tile scheduler (psa_sched.h): for the
+// masked scheme (paper Sec. 5) column tiles beyond the diagonal are absent from every loop in this
+// file -- not loaded, not multiplied, not exponentiated -- and only the block on the diagonal carries
+// an element predicate.
+//
+// Work items (one per pair of row tiles of one head) are listed heaviest first inside L2-sized groups
+// of heads; a CTA takes its first item by its index and every further one from a device counter, so
+// the list is consumed longest-processing-time-first whatever the items' run times turn out to be
+// (the role of the paper's pairing of long rows with short ones, Sec. 5.2: balance).  Because the CTA
+// lives on, the operand rings, the barriers' phases and the TMEM allocation carry over from item to
+// item: the next item's K, V and Q tiles are requested while the current item's last blocks are still
+// in the softmax, and its first scores are computed while the other row tile's output is written.
+//
+// CTA layout (576 threads): warp 0 = scheduler + TMA producer, warp 1 = MMA issuer, warps 2-9 = softmax
+// and epilogue of row tile 0, warps 10-17 = the same for row tile 1.  Within a tile's eight warps,
+// warp pairs (w, w+4) share a TMEM lane quarter (32 rows) and split the 128 columns of S in halves;
+// the pair agrees on the row maximum through shared memory.
+// TMEM columns, d = 128: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_t (bf16, two per
+// column) overlays S_t: keys 0-63 at S_t columns [0,32), keys 64-127 at [64,96), each written by the
+// thread that owns that half of the row.  d = 64: S0 S1 | P0 P1 [256,384) | O0 O1 [384,512): P has
+// its own columns, so S of the next key block is computed while the softmax of the current one runs.
+#include "psa_internal.h"
+#include "psa_sched.h"
+#include "psa_softmax.cuh"
+#include "psa_tma.h"
+#include "sm100.cuh"
+
+namespace psa {
+
+namespace {
+
+template <int D>
+struct PCfg {
+    static constexpr int SUB = D / 64;                  // 64-column sub-tiles per 128-row tile
+    static constexpr int TILE_BYTES = 128 * D * 2;      // one Q, K or V tile
+    static constexpr int KSTAGES = D == 128 ? 2 : 4;
+    static constexpr int VSTAGES = D == 128 ? 2 : 4;
+    static constexpr int SMEM = (2 + KSTAGES + VSTAGES) * TILE_BYTES + 1024;
+    static constexpr bool SEP_P = D == 64;
+    static constexpr int TMEM_S = 0, TMEM_P = 256, TMEM_O = SEP_P ? 384 : 256;
+    static constexpr int POLY_OF_4 = PSA_POLY_OF_4;
+};
+
+struct PMaps {
+    CUtensorMap q, k, v;
+};
+
+struct PBars {
+    uint64_t item_full[2], item_empty[2];
+    uint64_t q_full[2], q_empty[2];
+    uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
+    uint64_t s_full[2], s_free[2], p_ready[2], o_done[2];
+};
+
+constexpr int ITEM_READERS = 1 + 2 * SOFTMAX_WARPS_PER_TILE;   // MMA issuer + one lane per softmax warp
+
+template <int D>
+__global__ void __launch_bounds__(ATTN_THREADS, 1)
+attn_persist_kernel(const __grid_constant__ PMaps maps, __nv_bfloat16* __restrict__ out, int n, int H, int scheme,
+                    int nbh, int group, int nitems, float sl2, DeviceCounters* dc) {
+    using Cfg = PCfg<D>;
+    constexpr bool SEP = Cfg::SEP_P;
+    constexpr int KST = Cfg::KSTAGES, VST = Cfg::VSTAGES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sQ = smem;                                          // 2 tiles
+    uint8_t* sK = sQ + 2 * Cfg::TILE_BYTES;                      // KSTAGES tiles
+    uint8_t* sV = sK + KST * Cfg::TILE_BYTES;                    // VSTAGES tiles
+    __shared__ PBars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_flag;
+    __shared__ int item_ring[2];
+    __shared__ float xch_max[2][2][2][128];   // [block parity][tile][column half][row]
+    __shared__ float xch_sum[2][2][128];      // [tile][column half][row]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int T = row_tiles(n);
+    const int masked = scheme == PSA_MASKED;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&bars.item_full[t], 1);
+            mbar_init(&bars.item_empty[t], ITEM_READERS);
+            mbar_init(&bars.q_full[t], 1);
+            mbar_init(&bars.q_empty[t], 1);
+            mbar_init(&bars.s_full[t], 1);
+            mbar_init(&bars.s_free[t], 32 * SOFTMAX_WARPS_PER_TILE);
+            mbar_init(&bars.p_ready[t], 32 * SOFTMAX_WARPS_PER_TILE);
+            mbar_init(&bars.o_done[t], 1);
+        }
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(&bars.k_full[s], 1); mbar_init(&bars.k_empty[s], 1);
+            mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 1) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    volatile int* abortp = &abort_flag;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ scheduler + TMA producer
+            // kc, vc: K and V tiles requested so far (ring position); qc[t]: loads of Q buffer t so far.
+            uint32_t kc = 0, vc = 0, qc[2] = {0, 0};
+            int idx = blockIdx.x;          // the grid never exceeds the item count
+            bool ok = true;
+            for (uint32_t it = 0; ok; ++it) {
+                const int slot = it & 1;
+                if (it >= 2) ok = mbar_wait(&bars.item_empty[slot], ((it >> 1) - 1) & 1, abortp);
+                if (!ok) break;
+                item_ring[slot] = idx < nitems ? idx : -1;
+                mbar_arrive(&bars.item_full[slot]);
+                if (idx >= nitems) break;
+                const CtaWork work = cta_work(idx, n, masked, nbh, group);
+                // the next item's index is fetched now, long before it is needed
+                const int next = (int)gridDim.x + (int)atomicAdd(&dc->next_item, 1u);
+                const int b = work.bh / H, h = work.bh - b * H;
+                const int col0 = h * D;
+                const int nkv0 = kv_tiles(work.tile0, T, scheme);
+                const int nkv1 = work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0;
+                const int maxkv = max(nkv0, nkv1);
+                for (int j = 0; j < maxkv && ok; ++j) {
+                    {
+                        const int s = kc % KST;
+                        if (kc >= (uint32_t)KST) ok = mbar_wait(&bars.k_empty[s], ((kc / KST) - 1) & 1, abortp);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&bars.k_full[s], Cfg::TILE_BYTES);
+                        for (int u = 0; u < Cfg::SUB; ++u)
+                            tma_load_3d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], col0 + 64 * u,
+                                        j * TILE, b);
+                        ++kc;
+                    }
+                    if (j == 0) {
+                        for (int t = 0; t < work.ntiles && ok; ++t) {
+                            if (qc[t] > 0) ok = mbar_wait(&bars.q_empty[t], (qc[t] - 1) & 1, abortp);
+                            if (!ok) break;
+                            mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
+                            for (int u = 0; u < Cfg::SUB; ++u)
+                                tma_load_3d(sQ + t * Cfg::TILE_BYTES + u * 16384, &maps.q, &bars.q_full[t],
+                                            col0 + 64 * u, (work.tile0 + t) * TILE, b);
+                            ++qc[t];
+                        }
+                        if (!ok) break;
+                    }
+                    {
+                        const int s = vc % VST;
+                        if (vc >= (uint32_t)VST) ok = mbar_wait(&bars.v_empty[s], ((vc / VST) - 1) & 1, abortp);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
+                        for (int u = 0; u < Cfg::SUB; ++u)
+                            tma_load_3d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], col0 + 64 * u,
+                                        j * TILE, b);
+                        ++vc;
+                    }
+                }
+                idx = next;
+            }
+            if (*abortp) {  // let copies already issued land before shared memory is released
+                for (int t = 0; t < 2; ++t)
+                    if (qc[t] > 0) mbar_wait_drain(&bars.q_full[t], (qc[t] - 1) & 1);
+                for (uint32_t c = kc > (uint32_t)KST ? kc - KST : 0; c < kc; ++c)
+                    mbar_wait_drain(&bars.k_full[c % KST], (c / KST) & 1);
+                for (uint32_t c = vc > (uint32_t)VST ? vc - VST : 0; c < vc; ++c)
+                    mbar_wait_drain(&bars.v_full[c % VST], (c / VST) & 1);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ MMA issuer
+            // Each row tile's blocks form a chain S_0, PV_0, S_1, PV_1, ...  The two tiles' chains are issued
+            // alternately: while the softmax warps of one tile work on their scores, the tensor pipe runs the
+            // other tile's MMAs, and it is this half-step offset that keeps the pipe busy.
+            //  * P over S (d = 128): PV_j and S_{j+1} of a tile go back to back under one commit, and the thread
+            //    sleeps on what each link needs, tile 0 then tile 1 then tile 0 ...
+            //  * P apart from S (d = 64): S_{j+1} needs only that S_j has been read, PV_j needs P_j; the two
+            //    tiles' events arrive in no fixed order, so the barriers are tested without blocking and
+            //    whatever has become possible is issued.
+            const uint32_t idescS = umma_idesc_bf16(128, 128, UMMA_K_MAJOR, UMMA_K_MAJOR);
+            const uint32_t idescO = umma_idesc_bf16(128, D, UMMA_K_MAJOR, UMMA_MN_MAJOR);
+            unsigned long long qk_blocks = 0, pv_blocks = 0;
+            const uint32_t q_lo[2] = {umma_desc_lo_kmajor(smem_u32(sQ)), umma_desc_lo_kmajor(smem_u32(sQ + Cfg::TILE_BYTES))};
+            const uint32_t k_lo = umma_desc_lo_kmajor(smem_u32(sK));
+            const uint32_t v_lo = umma_desc_lo_mnmajor(smem_u32(sV), 16384);
+            const uint32_t tS0 = tmem + Cfg::TMEM_S, tO0 = tmem + Cfg::TMEM_O;
+            uint32_t kbase = 0, vbase = 0;      // ring positions of the current item's first K and V tile
+            uint32_t parts[2] = {0, 0};         // earlier items in which tile slot t had rows
+            uint32_t blk0[2] = {0, 0};          // blocks of tile slot t in all earlier items
+            bool ok = true;
+            // S_t = Q_t K^T with K at ring position kc (phase 1, Eq. 1): D/16 MMAs of 128x128x16.
+            auto mma_S = [&](int t, uint32_t kc) {
+                const uint32_t q = q_lo[t], k = k_lo + (kc % KST) * (Cfg::TILE_BYTES >> 4);
+                const uint32_t dS = tS0 + t * 128;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = ((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
+                    umma_ss(dS, umma_desc_join(q + off, UMMA_DESC_HI_SW128), umma_desc_join(k + off, UMMA_DESC_HI_SW128),
+                            idescS, kk != 0);
+                }
+                ++qk_blocks;
+            };
+            // O_t (+)= P_t V with V at ring position vc (phase 3, Eq. 3): 8 MMAs of 128 x D x 16.
+            auto mma_PV = [&](int t, uint32_t vc, bool first) {
+                const uint32_t v = v_lo + (vc % VST) * (Cfg::TILE_BYTES >> 4);
+                const uint32_t dO = tO0 + t * D;
+                const uint32_t aP = SEP ? tmem + Cfg::TMEM_P + t * 64 : tS0 + t * 128;
+                if (first) {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(dO, aP + (SEP ? kk * 8 : (kk >> 2) * 64 + (kk & 3) * 8),
+                                umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, kk != 0);
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(dO, aP + (SEP ? kk * 8 : (kk >> 2) * 64 + (kk & 3) * 8),
+                                umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, 1);
+                }
+                ++pv_blocks;
+            };
+            for (uint32_t it = 0; ok; ++it) {
+                ok = mbar_wait(&bars.item_full[it & 1], (it >> 1) & 1, abortp);
+                if (!ok) break;
+                const int idx = item_ring[it & 1];
+                mbar_arrive(&bars.item_empty[it & 1]);
+                if (idx < 0) break;
+                const CtaWork work = cta_work(idx, n, masked, nbh, group);
+                const int nkv[2] = {kv_tiles(work.tile0, T, scheme),
+                                    work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0};
+                const int maxkv = max(nkv[0], nkv[1]);
+                if (!SEP) {
+                    // first scores of both tiles
+                    ok = mbar_wait(&bars.k_full[kbase % KST], (kbase / KST) & 1, abortp);
+                    for (int t = 0; t < work.ntiles && ok; ++t) {
+                        ok = mbar_wait(&bars.q_full[t], parts[t] & 1, abortp);
+                        if (!ok) break;
+                        tc_fence_after();
+                        mma_S(t, kbase);
+                        umma_commit(&bars.s_full[t]);
+                        if (nkv[t] == 1) umma_commit(&bars.q_empty[t]);
+                    }
+                    if (!ok) break;
+                    umma_commit(&bars.k_empty[kbase % KST]);
+                    for (int j = 0; j < maxkv && ok; ++j) {
+                        for (int t = 0; t < work.ntiles && ok; ++t) {
+                            if (j >= nkv[t]) continue;
+                            const uint32_t vc = vbase + j, kc = kbase + j + 1;
+                            const bool has_next = j + 1 < nkv[t];
+                            // operand tiles first: these are normally long complete and cost only the poll
+                            ok = mbar_wait(&bars.v_full[vc % VST], (vc / VST) & 1, abortp);
+                            if (ok && has_next) ok = mbar_wait(&bars.k_full[kc % KST], (kc / KST) & 1, abortp);
+                            if (ok) ok = mbar_wait(&bars.p_ready[t], (blk0[t] + j) & 1, abortp);
+                            if (!ok) break;
+                            tc_fence_after();
+                            mma_PV(t, vc, j == 0);
+                            if (has_next) mma_S(t, kc);
+                            umma_commit(&bars.o_done[t]);
+                            // an operand tile is released behind its last user in this fixed order
+                            const bool last_v = t == work.ntiles - 1 || j >= nkv[t + 1];
+                            if (last_v) umma_commit(&bars.v_empty[vc % VST]);
+                            if (has_next) {
+                                if (t == work.ntiles - 1 || j + 1 >= nkv[t + 1]) umma_commit(&bars.k_empty[kc % KST]);
+                                if (j + 1 == nkv[t] - 1) umma_commit(&bars.q_empty[t]);
+                            }
+                        }
+                    }
+                } else {
+                    int nS[2] = {0, 0}, nPV[2] = {0, 0};     // S and PV blocks issued for each tile in this item
+                    uint64_t t_last = 0;
+                    uint32_t idle = 0;
+                    // the K (V) tile at block j is released by whichever tile issues its S_j (PV_j) last
+                    auto k_last_user = [&](int t, int j) { const int o = t ^ 1; return j >= nkv[o] || nS[o] > j; };
+                    auto v_last_user = [&](int t, int j) { const int o = t ^ 1; return j >= nkv[o] || nPV[o] > j; };
+                    while (ok && (nPV[0] < nkv[0] || nPV[1] < nkv[1])) {
+                        bool progressed = false;
+                        for (int t = 0; t < work.ntiles; ++t) {
+                            int j = nS[t];
+                            if (j < nkv[t]) {
+                                const uint32_t kc = kbase + j, sidx = blk0[t] + j;
+                                bool rdy = mbar_test(&bars.k_full[kc % KST], (kc / KST) & 1);
+                                if (rdy && j == 0) rdy = mbar_test(&bars.q_full[t], parts[t] & 1);
+                                // the softmax warps must have taken the previous scores of this tile out of TMEM
+                                if (rdy && sidx > 0) rdy = mbar_test(&bars.s_free[t], (sidx - 1) & 1);
+                                if (rdy) {
+                                    tc_fence_after();
+                                    mma_S(t, kc);
+                                    umma_commit(&bars.s_full[t]);
+                                    ++nS[t];
+                                    if (k_last_user(t, j)) umma_commit(&bars.k_empty[kc % KST]);
+                                    if (j == nkv[t] - 1) umma_commit(&bars.q_empty[t]);
+                                    progressed = true;
+                                }
+                            }
+                            j = nPV[t];
+                            if (j < nkv[t] && j < nS[t]) {
+                                const uint32_t vc = vbase + j;
+                                bool rdy = mbar_test(&bars.p_ready[t], (blk0[t] + j) & 1);
+                                if (rdy) rdy = mbar_test(&bars.v_full[vc % VST], (vc / VST) & 1);
+                                if (rdy) {
+                                    tc_fence_after();
+                                    mma_PV(t, vc, j == 0);
+                                    umma_commit(&bars.o_done[t]);
+                                    ++nPV[t];
+                                    if (v_last_user(t, j)) umma_commit(&bars.v_empty[vc % VST]);
+                                    progressed = true;
+                                }
+                            }
+                        }
+                        if (progressed) {
+                            idle = 0;
+                        } else if ((++idle & 255u) == 0u) {
+                            if (*abortp) ok = false;
+                            else if (idle == 256u) t_last = globaltimer_ns();
+                            else if (globaltimer_ns() - t_last > 4 * PSA_WAIT_LIMIT_NS) { *abortp = 1; ok = false; }
+                        }
+                    }
+                }
+                kbase += maxkv;
+                vbase += maxkv;
+                for (int t = 0; t < work.ntiles; ++t) { ++parts[t]; blk0[t] += nkv[t]; }
+            }
+            const unsigned long long block_macs = (unsigned long long)TILE * TILE * D;
+            if (qk_blocks) atomicAdd(&dc->qk_macs, qk_blocks * block_macs);
+            if (pv_blocks) {
+                atomicAdd(&dc->pv_macs, pv_blocks * block_macs);
+                atomicAdd(&dc->exps, pv_blocks * (unsigned long long)(TILE * TILE));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax + epilogue
+        // TPR threads share a query row; thread `part` owns block columns [part*CPT, (part+1)*CPT).
+        constexpr int CPT = 128 / TPR;                           // score columns per thread
+        constexpr int NCH = CPT / 32;                            // 32-column chunks per thread
+        constexpr int OPT = D / TPR;                             // output columns per thread
+        const int sw = warp - CTRL_WARPS;
+        const int t = sw / SOFTMAX_WARPS_PER_TILE;              // row tile slot of this warp
+        const int part = (sw % SOFTMAX_WARPS_PER_TILE) >> 2;    // which share of the row's columns
+        const int q = warp & 3;                                 // TMEM lane quarter this warp may access
+        const int r = q * 32 + lane;                            // row inside the tile = TMEM lane
+        const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
+        const uint32_t tS = tmem + Cfg::TMEM_S + t * 128 + lane_off;
+        const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off + part * OPT;
+        const uint32_t tP = tmem + Cfg::TMEM_P + t * 64 + lane_off;     // separate-P layout only
+        const int pair_bar = 1 + t * 4 + q;                     // named barrier of the warps sharing rows
+        const int tile_bar = 9 + t;                             // named barrier of all softmax warps of the tile
+        const int col_base = part * CPT;
+        const size_t out_pitch = (size_t)H * D;                 // elements between output rows
+        uint32_t my_items = 0;                                  // items this tile slot took part in
+        uint32_t blk = 0;                                       // blocks this tile slot has processed, all items
+        bool ok = true;
+        for (uint32_t it = 0; ok; ++it) {
+            ok = mbar_wait(&bars.item_full[it & 1], (it >> 1) & 1, abortp);
+            // all warps of the tile slot take the item or none does (one may have given up the wait)
+            ok = named_bar_all(ok, tile_bar, 32 * SOFTMAX_WARPS_PER_TILE);
+            if (!ok) break;
+            const int idx = item_ring[it & 1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars.item_empty[it & 1]);
+            if (idx < 0) break;
+            const CtaWork work = cta_work(idx, n, masked, nbh, group);
+            if (t >= work.ntiles) continue;
+            const int b = work.bh / H, h = work.bh - b * H;
+            const int It = work.tile0 + t;
+            const int nkv = kv_tiles(It, T, scheme);
+            float m_run = -INFINITY, l_run = 0.f;
+            for (int j = 0; j < nkv; ++j, ++blk) {
+                if (SEP) {
+                    ok = mbar_wait(&bars.s_full[t], blk & 1, abortp);                 // every S has its own commit
+                } else {
+                    // block 0 waits for the item's first S; later blocks for the commit behind PV_{j-1} and S_j
+                    if (j == 0) ok = mbar_wait(&bars.s_full[t], my_items & 1, abortp);
+                    else ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                if (TPR == 1 && !ok) break;
+                // Element predicate: on the diagonal block of the masked scheme keys beyond the row's own index,
+                // and on a ragged last block keys beyond the sequence, carry no weight.  `cb` = last kept column.
+                const int nvalid = min(TILE, n - j * TILE);
+                const bool on_diag = masked && (j == It);
+                const bool diag = on_diag || nvalid < TILE;
+                const int cb = min(on_diag ? r : TILE - 1, nvalid - 1);
+                float mx = -INFINITY;
+                uint32_t sreg[NCH][32];
+                if (ok) {
+                    // ---- pass 1: maximum of this thread's scores
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) tmem_ld32(tS + col_base + 32 * c, sreg[c]);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c)
+                        mx = diag ? max_chunk32<true>(sreg[c], col_base + 32 * c, cb, mx)
+                                  : max_chunk32<false>(sreg[c], col_base + 32 * c, r, mx);
+                }
+                if (TPR == 2) {
+                    // The two threads of a row meet here to exchange their half-row maxima (and to leave
+                    // together if either gave up a wait).
+                    xch_max[blk & 1][t][part][r] = mx;
+                    ok = named_bar_all(ok, pair_bar, 64);
+                    if (!ok) break;
+                    mx = fmaxf(mx, xch_max[blk & 1][t][part ^ 1][r]);
+                }
+                const float mx2 = mx * sl2;
+                float alpha = 1.f;
+                if (mx2 > m_run + RESCALE_THRESHOLD) {   // also taken on the first block (m_run = -inf)
+                    alpha = ex2_mufu(m_run - mx2);
+                    m_run = mx2;
+                }
+                // ---- pass 2: P = exp2(S*sl2 - m) as bf16
+                float rowsum = 0.f;
+                if (TPR == 2) {      // the scores were only reduced so far: fetch them again
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) tmem_ld32(tS + col_base + 32 * c, sreg[c]);
+                    tc_wait_ld();
+                }
+                if (SEP) {
+                    // S is in registers: the issuer may overwrite it with the next scores while the exponentials run
+                    tc_fence_before();
+                    mbar_arrive(&bars.s_free[t]);
+                    // P and O are still in use by PV_{j-1} until its commit.  A wait given up here is not
+                    // acted on before the next pair barrier, so that the two threads of a row stay together.
+                    if (j > 0) {
+                        ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
+                        ok = __all_sync(0xffffffffu, ok);
+                        tc_fence_after();
+                    }
+                }
+                if (ok) {
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        uint32_t pk[16];
+                        const int kc = col_base + 32 * c;            // first key column of the chunk
+                        rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(sreg[c], sl2, -m_run, kc, cb, pk)
+                                       : exp_chunk32<Cfg::POLY_OF_4, false>(sreg[c], sl2, -m_run, kc, r, pk);
+                        // P over S: keys [kc, kc+32) go to S columns (kc/64)*64 + (kc%64)/2, behind this thread's own reads
+                        tmem_st16(SEP ? tP + (kc >> 1) : tS + (kc >> 6) * 64 + ((kc & 63) >> 1), pk);
+                    }
+                }
+                l_run = fmaf(l_run, alpha, rowsum);
+                if (ok && j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8
+#pragma unroll
+                    for (int c = 0; c < OPT / 32; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tO + 32 * c, v);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                        tmem_st32(tO + 32 * c, v);
+                    }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(&bars.p_ready[t]);
+            }
+            if (ok) ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
+            if (TPR == 2) xch_sum[t][part][r] = l_run;
+            ok = named_bar_all(ok, tile_bar, 32 * SOFTMAX_WARPS_PER_TILE);
+            if (!ok) break;
+            // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row), straight from
+            // TMEM to global memory: each thread holds OPT consecutive columns of its own row.
+            tc_fence_after();
+            const float inv = 1.f / (TPR == 2 ? l_run + xch_sum[t][part ^ 1][r] : l_run);
+            const int row = It * TILE + r;
+            __nv_bfloat16* dst = out + ((size_t)b * n + row) * out_pitch + (size_t)h * D + part * OPT;
+#pragma unroll
+            for (int c = 0; c < OPT / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tO + 32 * c, v);
+                tc_wait_ld();
+                if (row < n) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint4 o;
+                        o.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]) * inv, __uint_as_float(v[g * 8 + 1]) * inv);
+                        o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]) * inv, __uint_as_float(v[g * 8 + 3]) * inv);
+                        o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]) * inv, __uint_as_float(v[g * 8 + 5]) * inv);
+                        o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]) * inv, __uint_as_float(v[g * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4*>(dst + 32 * c + 8 * g) = o;
+                    }
+                }
+            }
+            // (the next write to O_t, PV_0 of the tile's next item, waits for P of that item, which every
+            // thread of the tile signals only after these reads)
+            tc_fence_before();
+            ++my_items;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicExch(&dc->status, (int)PSA_ERR_TIMEOUT);
+    if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+template <int D>
+int launch_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, float scale,
+                   int scheme, DeviceCounters* dc, cudaStream_t stream) {
+    using Cfg = PCfg<D>;
+    static bool attr_set = false;
+    static int sm_count = 0;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(attn_persist_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
+        int dev = 0;
+        if (e == cudaSuccess) e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess || sm_count <= 0) { set_cuda_error(e, "attention kernel set-up"); return PSA_ERR_CUDA; }
+        attr_set = true;
+    }
+    const uint64_t cols = (uint64_t)H * D;
+    PMaps maps;
+    if (!make_tensor_map_bf16_3d(&maps.q, Q, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.k, K, B, n, cols, 128) ||
+        !make_tensor_map_bf16_3d(&maps.v, V, B, n, cols, 128))
+        return PSA_ERR_CUDA;
+    const long long nitems = (long long)B * H * ctas_per_head(n);
+    if (nitems > 0x7fffffffLL - sm_count) return PSA_ERR_SHAPE;
+    const int grid = (int)(nitems < sm_count ? nitems : sm_count);
+    attn_persist_kernel<D><<<grid, ATTN_THREADS, Cfg::SMEM, stream>>>(
+        maps, static_cast<__nv_bfloat16*>(out), n, H, scheme, B * H, lpt_group(scheme, B * H, n, D), (int)nitems,
+        scale * LOG2E, dc);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error(e, "attn_persist_kernel launch"); return PSA_ERR_CUDA; }
+    return PSA_OK;
+}
+
+}  // namespace
+
+// FULL and MASKED schemes.  `dc->next_item` must be zero when the kernel starts (the per-call clearing of the
+// counter block does that); the kernel is launched once per call.
+int bf16_attention_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, int d,
+                           float scale, int scheme, DeviceCounters* dc, cudaStream_t stream) {
+    if (scheme != PSA_FULL && scheme != PSA_MASKED) return PSA_ERR_SCHEME_ARGS;
+    if (d == 64) return launch_persist<64>(Q, K, V, out, B, H, n, scale, scheme, dc, stream);
+    if (d == 128) return launch_persist<128>(Q, K, V, out, B, H, n, scale, scheme, dc, stream);
+    return PSA_ERR_UNSUPPORTED;
+}
+
+}  // namespace psa

@@ -15,7 +15,7 @@ struct DeviceCounters {
     unsigned long long pv_macs;
     unsigned long long exps;
     int status;  // PSA_OK or PSA_ERR_TIMEOUT
-    int pad;
+    unsigned int next_item;  // work-list cursor of the persistent attention kernel
 };
 
 // ---- fp32 CUDA-core path (psa_f32.cu) ----
@@ -34,6 +34,9 @@ int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int n
 int bf16_attention(const void* Q, const void* K, const void* V, void* out, float* S, size_t s_bytes, int B,
                    int H, int n, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
 size_t bf16_symmetric_scratch_bytes(int B, int H, int n);
+// The persistent fused kernel behind bf16_attention for PSA_FULL and PSA_MASKED (psa_attn_persist.cu).
+int bf16_attention_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, int d,
+                           float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
 
 void set_cuda_error(cudaError_t e, const char* where);
 void set_error_text(const char* text);
