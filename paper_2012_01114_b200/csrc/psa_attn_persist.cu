@@ -46,14 +46,18 @@ struct PCfg {
     static constexpr int TILE_BYTES = 128 * D * 2;      // one Q, K or V tile
     static constexpr int KSTAGES = D == 128 ? 2 : 4;
     static constexpr int VSTAGES = D == 128 ? 2 : 4;
-    static constexpr int SMEM = (2 + KSTAGES + VSTAGES) * TILE_BYTES + 1024;
+    // output staging buffers of 32 rows x D columns: one for each of an item's 8 units (d = 64), 3 that the units
+    // take in turn (d = 128, where shared memory has no room for more)
+    static constexpr int STAGE_BYTES = 32 * D * 2;
+    static constexpr int STAGE_BUFS = D == 64 ? 8 : 3;
+    static constexpr int SMEM = (2 + KSTAGES + VSTAGES) * TILE_BYTES + STAGE_BUFS * STAGE_BYTES + 1024;
     static constexpr bool SEP_P = D == 64;
     static constexpr int TMEM_S = 0, TMEM_P = 256, TMEM_O = SEP_P ? 384 : 256;
     static constexpr int POLY_OF_4 = PSA_POLY_OF_4;
 };
 
 struct PMaps {
-    CUtensorMap q, k, v;
+    CUtensorMap q, k, v, o;
 };
 
 struct PBars {
@@ -63,12 +67,27 @@ struct PBars {
     uint64_t s_full[2], s_free[2], p_ready[2], o_done[2];
 };
 
+// Bounded wait until a shared-memory counter, which only grows, has reached `target`.
+__device__ __forceinline__ bool count_wait(const volatile uint32_t* counter, uint32_t target, volatile int* abort_flag) {
+    if (*counter >= target) return true;
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t it = 0;
+    while (*counter < target) {
+        __nanosleep(20);
+        if ((++it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (globaltimer_ns() - t0 > PSA_WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+        }
+    }
+    return true;
+}
+
 constexpr int ITEM_READERS = 1 + 2 * SOFTMAX_WARPS_PER_TILE;   // MMA issuer + one lane per softmax warp
 
 template <int D>
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
-attn_persist_kernel(const __grid_constant__ PMaps maps, __nv_bfloat16* __restrict__ out, int n, int H, int scheme,
-                    int nbh, int group, int nitems, float sl2, DeviceCounters* dc) {
+attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme, int nbh,
+                    int group, int nitems, float sl2, DeviceCounters* dc) {
     using Cfg = PCfg<D>;
     constexpr bool SEP = Cfg::SEP_P;
     constexpr int KST = Cfg::KSTAGES, VST = Cfg::VSTAGES;
@@ -77,10 +96,12 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, __nv_bfloat16* __restric
     uint8_t* sQ = smem;                                          // 2 tiles
     uint8_t* sK = sQ + 2 * Cfg::TILE_BYTES;                      // KSTAGES tiles
     uint8_t* sV = sK + KST * Cfg::TILE_BYTES;                    // VSTAGES tiles
+    uint8_t* sStage = sV + VST * Cfg::TILE_BYTES;                // STAGE_BUFS output staging tiles
     __shared__ PBars bars;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
     __shared__ int item_ring[2];
+    __shared__ volatile uint32_t stage_released[8];   // per staging buffer: uses whose store has read it
     __shared__ float xch_max[2][2][2][128];   // [block parity][tile][column half][row]
     __shared__ float xch_sum[2][2][128];      // [tile][column half][row]
 
@@ -90,6 +111,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, __nv_bfloat16* __restric
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
+        for (int i = 0; i < 8; ++i) stage_released[i] = 0;
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bars.item_full[t], 1);
             mbar_init(&bars.item_empty[t], ITEM_READERS);
@@ -356,23 +378,30 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, __nv_bfloat16* __restric
         const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off + part * OPT;
         const uint32_t tP = tmem + Cfg::TMEM_P + t * 64 + lane_off;     // separate-P layout only
         const int pair_bar = 1 + t * 4 + q;                     // named barrier of the warps sharing rows
-        const int tile_bar = 9 + t;                             // named barrier of all softmax warps of the tile
         const int col_base = part * CPT;
-        const size_t out_pitch = (size_t)H * D;                 // elements between output rows
         uint32_t my_items = 0;                                  // items this tile slot took part in
         uint32_t blk = 0;                                       // blocks this tile slot has processed, all items
         bool ok = true;
-        for (uint32_t it = 0; ok; ++it) {
-            ok = mbar_wait(&bars.item_full[it & 1], (it >> 1) & 1, abortp);
-            // all warps of the tile slot take the item or none does (one may have given up the wait)
-            ok = named_bar_all(ok, tile_bar, 32 * SOFTMAX_WARPS_PER_TILE);
+        for (uint32_t it = 0;; ++it) {
+            if (ok) ok = mbar_wait(&bars.item_full[it & 1], (it >> 1) & 1, abortp);
+            // the two warps that share rows take the item or neither does (one may have given up a wait); pairs of
+            // a slot are not held together here: a pair whose output is on its way starts on the next item
+            ok = named_bar_all(ok, pair_bar, 32 * TPR);
             if (!ok) break;
             const int idx = item_ring[it & 1];
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars.item_empty[it & 1]);
             if (idx < 0) break;
             const CtaWork work = cta_work(idx, n, masked, nbh, group);
-            if (t >= work.ntiles) continue;
+            if (t >= work.ntiles) {
+                // no rows for this slot in this item: its units' turns at the staging buffers are passed on
+                if (part == 0 && lane == 0) {
+                    const uint32_t unit = it * 8u + 4u * t + q;
+                    const uint32_t sbuf = unit % Cfg::STAGE_BUFS, suse = unit / Cfg::STAGE_BUFS;
+                    if (count_wait(&stage_released[sbuf], suse, abortp)) stage_released[sbuf] = suse + 1;
+                }
+                continue;
+            }
             const int b = work.bh / H, h = work.bh - b * H;
             const int It = work.tile0 + t;
             const int nkv = kv_tiles(It, T, scheme);
@@ -468,20 +497,26 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, __nv_bfloat16* __restric
             }
             if (ok) ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
             if (TPR == 2) xch_sum[t][part][r] = l_run;
-            ok = named_bar_all(ok, tile_bar, 32 * SOFTMAX_WARPS_PER_TILE);
+            ok = named_bar_all(ok, pair_bar, 32 * TPR);
             if (!ok) break;
-            // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row), straight from
-            // TMEM to global memory: each thread holds OPT consecutive columns of its own row.
+            // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row), bf16.  The two warps
+            // that share 32 rows write them into a staging buffer (32 rows x D columns) and one lane hands
+            // it to TMA.  Buffers are taken in the fixed order of the units (item, slot, lane quarter); a unit
+            // waits until the store of the unit that last used its buffer has read it.
             tc_fence_after();
             const float inv = 1.f / (TPR == 2 ? l_run + xch_sum[t][part ^ 1][r] : l_run);
-            const int row = It * TILE + r;
-            __nv_bfloat16* dst = out + ((size_t)b * n + row) * out_pitch + (size_t)h * D + part * OPT;
+            const uint32_t unit = it * 8u + 4u * t + q;
+            const uint32_t sbuf = unit % Cfg::STAGE_BUFS, suse = unit / Cfg::STAGE_BUFS;
+            uint8_t* stage = sStage + sbuf * Cfg::STAGE_BYTES;
+            ok = count_wait(&stage_released[sbuf], suse, abortp);
+            if (ok) {
 #pragma unroll
-            for (int c = 0; c < OPT / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tO + 32 * c, v);
-                tc_wait_ld();
-                if (row < n) {
+                for (int c = 0; c < OPT / 32; ++c) {
+                    const int col = part * OPT + 32 * c;            // first of 32 output columns handled here
+                    uint32_t v[32];
+                    tmem_ld32(tO + 32 * c, v);
+                    tc_wait_ld();
+                    uint8_t* sub = stage + (col / 64) * 4096;       // [32 rows x 64 columns] sub-tiles, 128-byte swizzle
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         uint4 o;
@@ -489,9 +524,20 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, __nv_bfloat16* __restric
                         o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]) * inv, __uint_as_float(v[g * 8 + 3]) * inv);
                         o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]) * inv, __uint_as_float(v[g * 8 + 5]) * inv);
                         o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]) * inv, __uint_as_float(v[g * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(dst + 32 * c + 8 * g) = o;
+                        *reinterpret_cast<uint4*>(sub + swz128_offset(lane, (col % 64) / 8 + g)) = o;
                     }
                 }
+                fence_async_smem();
+            }
+            // (a pair that gave up carries that into the vote at the top of the next item)
+            ok = named_bar_all(ok, pair_bar, 32 * TPR);
+            if (ok && part == 0 && lane == 0) {
+                for (int u = 0; u < Cfg::SUB; ++u)
+                    tma_store_3d(&maps.o, stage + u * 4096, h * D + 64 * u, It * TILE + q * 32, b);
+                tma_store_commit();
+                tma_store_wait_read();   // the buffer may be rewritten; the global writes complete on their own
+                __threadfence_block();
+                stage_released[sbuf] = suse + 1;
             }
             // (the next write to O_t, PV_0 of the tile's next item, waits for P of that item, which every
             // thread of the tile signals only after these reads)
@@ -522,13 +568,13 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
     const uint64_t cols = (uint64_t)H * D;
     PMaps maps;
     if (!make_tensor_map_bf16_3d(&maps.q, Q, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.k, K, B, n, cols, 128) ||
-        !make_tensor_map_bf16_3d(&maps.v, V, B, n, cols, 128))
+        !make_tensor_map_bf16_3d(&maps.v, V, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.o, out, B, n, cols, 32))
         return PSA_ERR_CUDA;
     const long long nitems = (long long)B * H * ctas_per_head(n);
     if (nitems > 0x7fffffffLL - sm_count) return PSA_ERR_SHAPE;
     const int grid = (int)(nitems < sm_count ? nitems : sm_count);
     attn_persist_kernel<D><<<grid, ATTN_THREADS, Cfg::SMEM, stream>>>(
-        maps, static_cast<__nv_bfloat16*>(out), n, H, scheme, B * H, lpt_group(scheme, B * H, n, D), (int)nitems,
+        maps, n, H, scheme, B * H, lpt_group(scheme, B * H, n, D), (int)nitems,
         scale * LOG2E, dc);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "attn_persist_kernel launch"); return PSA_ERR_CUDA; }
