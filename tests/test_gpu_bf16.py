@@ -80,6 +80,16 @@ def test_ragged_sequence_lengths(scheme, B, H, n, d):
     _check_census(B, H, n, 0, d, scheme)
 
 
+@pytest.mark.parametrize("scheme", [oracle.FULL, oracle.MASKED])
+@pytest.mark.parametrize("B,H,n,d", [(4, 40, 384, 64), (2, 80, 300, 128), (3, 100, 256, 128), (5, 64, 130, 64)])
+def test_more_work_items_than_sms(scheme, B, H, n, d):
+    # Several hundred (head, pair of row tiles) items: every CTA of the persistent kernel walks several of them,
+    # with an odd number of row tiles (a slot without rows in every other item) and ragged last blocks among them.
+    err = _core_case(B, H, n, d, scheme, seed=3 * n + d)
+    assert err <= TOL_BF16, err
+    _check_census(B, H, n, 0, d, scheme)
+
+
 def test_ragged_layer_with_projections():
     B, H, n, D, d = 2, 2, 300, 128, 64
     Xv, Xb = inputs.tensor(17, 0, (B, n, D), 1.0, "bf16")
