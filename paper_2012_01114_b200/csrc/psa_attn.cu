@@ -5,13 +5,17 @@
 // through memory:
 //
 //   sym_scores_kernel   phase 1, one CTA per unordered pair of 128-row tiles {I, J}, J <= I: the block
-//                       S_IJ = scale * X_I X_J^T on the tensor core, written ONCE to a scratch matrix at
-//                       block (I, J).  Blocks above the diagonal are neither computed nor stored.
-//   sym_attn_kernel     phases 2 and 3 per pair of row tiles: the row of blocks S_I,* is fetched by TMA into
-//                       shared memory -- block (I, J) as stored for J <= I, block (J, I) read transposed for
+//                       S_IJ = scale * X_I X_J^T on the tensor core, written ONCE to the scratch.  Blocks
+//                       above the diagonal are neither computed nor stored.
+//   sym_attn_kernel     phases 2 and 3 per pair of row tiles: the row of blocks S_I,* is fetched into shared
+//                       memory -- block (I, J) as stored for J <= I, block (J, I) read transposed for
 //                       J > I (the reuse) -- then softmax and O += P V as in the fused kernel of the other
 //                       schemes (two threads per row, P written to TMEM as bf16, V = X staged by TMA,
 //                       accumulator O in TMEM, the division of Eq. 2 applied once to the output row).
+//
+// The scratch holds, per head, the T(T+1)/2 blocks at or below the block diagonal, each as one contiguous
+// 64 KB image of its shared-memory form (four [128 rows x 32 fp32] sub-tiles in the 128-byte swizzle), so
+// that a block moves between shared and global memory as one bulk copy of consecutive bytes.
 //
 // The fused persistent kernel of the FULL and MASKED schemes is in psa_attn_persist.cu.
 #include "psa_internal.h"
@@ -26,6 +30,10 @@ namespace {
 
 constexpr int S_SUB_BYTES = 128 * 32 * 4;       // one [128 rows x 32 fp32] sub-tile of a score block, 128-byte rows
 constexpr int S_BLOCK_BYTES = 4 * S_SUB_BYTES;  // one 128 x 128 fp32 score block: 64 KB
+#ifndef PSA_SYM_COPIES
+#define PSA_SYM_COPIES 4
+#endif
+constexpr int S_COPIES = PSA_SYM_COPIES;        // bulk copies a block is moved in
 
 template <int D>
 struct SymCfg {
@@ -39,7 +47,6 @@ struct SymCfg {
 
 struct SymMaps {
     CUtensorMap x;     // X as [batch, n, H*d] bf16, boxes of 128 rows x 64 columns
-    CUtensorMap s;     // score scratch as [heads * npad, npad] fp32, boxes of 128 rows x 32 columns
     CUtensorMap o;     // output, like x
 };
 
@@ -54,7 +61,8 @@ struct SymBars {
 // formed: its readers take (I, J) transposed.
 template <int D>
 __global__ void __launch_bounds__(128)
-sym_scores_kernel(const __grid_constant__ SymMaps maps, int n, int H, int bh0, float scale, DeviceCounters* dc) {
+sym_scores_kernel(const __grid_constant__ SymMaps maps, float* __restrict__ Sg, int n, int H, int bh0, float scale,
+                  DeviceCounters* dc) {
     constexpr int SUB = D / 64, TILE_BYTES = 128 * D * 2;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -73,7 +81,7 @@ sym_scores_kernel(const __grid_constant__ SymMaps maps, int n, int H, int bh0, f
     sym_pair(blockIdx.x - hl * np, &I, &J);
     const int bh = bh0 + hl, b = bh / H, h = bh - b * H;
     const int col0 = h * D;
-    const int npad = T * TILE;                       // the scratch is padded to whole tiles
+    const int pair = blockIdx.x - hl * np;           // = I (I + 1) / 2 + J: the block's place in the head's scratch
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -113,7 +121,7 @@ sym_scores_kernel(const __grid_constant__ SymMaps maps, int n, int H, int bh0, f
     const bool ready = mbar_wait(&acc_bar, 0, abortp);
     if (__syncthreads_and(ready)) {
         // every MMA has read its operands: the block goes to shared memory as four [128 x 32] fp32 sub-tiles in
-        // the 128-byte swizzle, each thread its own row, and from there to the scratch by TMA
+        // the 128-byte swizzle, each thread its own row, and from there to the scratch as one bulk copy
         tc_fence_after();
         const int r = warp * 32 + lane;
 #pragma unroll 1
@@ -132,8 +140,9 @@ sym_scores_kernel(const __grid_constant__ SymMaps maps, int n, int H, int bh0, f
         fence_async_smem();
         __syncthreads();
         if (threadIdx.x == 0) {
-            for (int u = 0; u < 4; ++u)
-                tma_store_2d(&maps.s, sS + u * S_SUB_BYTES, J * TILE + 32 * u, hl * npad + I * TILE);
+            float* dst = Sg + ((size_t)hl * np + pair) * (S_BLOCK_BYTES / 4);
+            for (int u = 0; u < S_COPIES; ++u)
+                bulk_store_1d(dst + u * (S_BLOCK_BYTES / S_COPIES / 4), sS + u * (S_BLOCK_BYTES / S_COPIES), S_BLOCK_BYTES / S_COPIES);
             tma_store_commit();
             tma_store_wait_read();   // shared memory may be released; the writes complete on their own
         }
@@ -149,7 +158,8 @@ sym_scores_kernel(const __grid_constant__ SymMaps maps, int n, int H, int bh0, f
 // 10-17 = softmax and epilogue of row tile 0 / 1, two threads per row.
 template <int D>
 __global__ void __launch_bounds__(ATTN_THREADS, 1)
-sym_attn_kernel(const __grid_constant__ SymMaps maps, int n, int H, int bh0, int nbh, DeviceCounters* dc) {
+sym_attn_kernel(const __grid_constant__ SymMaps maps, const float* __restrict__ Sg, int n, int H, int bh0, int nbh,
+                DeviceCounters* dc) {
     using Cfg = SymCfg<D>;
     constexpr int VST = Cfg::VSTAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -164,7 +174,7 @@ sym_attn_kernel(const __grid_constant__ SymMaps maps, int n, int H, int bh0, int
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int T = row_tiles(n);
-    const int npad = T * TILE;
+    const int np = sym_pairs(T);
     const CtaWork work = cta_work(blockIdx.x, n, 0, nbh, 1);
     const int hl = work.bh;                              // head inside this pass
     const int bh = bh0 + hl;
@@ -203,9 +213,10 @@ sym_attn_kernel(const __grid_constant__ SymMaps maps, int n, int H, int bh0, int
                     const int It = work.tile0 + t;
                     const int bi = j <= It ? It : j, bj = j <= It ? j : It;      // stored block (row tile, column tile)
                     mbar_arrive_expect_tx(&bars.s_full[t], S_BLOCK_BYTES);
-                    for (int u = 0; u < 4; ++u)
-                        tma_load_2d(sS + t * S_BLOCK_BYTES + u * S_SUB_BYTES, &maps.s, &bars.s_full[t], bj * TILE + 32 * u,
-                                    hl * npad + bi * TILE);
+                    const float* src = Sg + ((size_t)hl * np + bi * (bi + 1) / 2 + bj) * (S_BLOCK_BYTES / 4);
+                    for (int u = 0; u < S_COPIES; ++u)      // several copies in flight move a block faster than one
+                        bulk_load_1d(sS + t * S_BLOCK_BYTES + u * (S_BLOCK_BYTES / S_COPIES), src + u * (S_BLOCK_BYTES / S_COPIES / 4),
+                                     S_BLOCK_BYTES / S_COPIES, &bars.s_full[t]);
                     ++s_loads[t];
                 }
                 if (!ok) break;
@@ -406,15 +417,18 @@ sym_attn_kernel(const __grid_constant__ SymMaps maps, int n, int H, int bh0, int
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
-constexpr size_t SYM_SCRATCH_CAP = size_t(2) << 30;  // bytes of score scratch per pass
+// Heads per pass: as many as the scratch cap allows, in passes of equal size (the scratch is reused from pass
+// to pass).  Passes small enough to stay in L2 were measured slower: the kernels of a small pass do not fill the GPU.
+constexpr size_t SYM_SCRATCH_CAP = size_t(2) << 30;   // bytes of score scratch per pass
 
 int sym_heads_per_pass(int B, int H, int n) {
-    const size_t npad = (size_t)row_tiles(n) * TILE;
-    const size_t per_head = npad * npad * sizeof(float);
+    const size_t per_head = (size_t)sym_pairs(row_tiles(n)) * S_BLOCK_BYTES;
+    const size_t all = (size_t)B * H;
     size_t hp = SYM_SCRATCH_CAP / per_head;
     if (hp < 1) hp = 1;
-    if (hp > (size_t)B * H) hp = (size_t)B * H;
-    return (int)hp;
+    if (hp > all) hp = all;
+    const size_t passes = (all + hp - 1) / hp;
+    return (int)((all + passes - 1) / passes);
 }
 
 template <int D>
@@ -432,17 +446,16 @@ int launch_symmetric(const void* X, void* out, float* S, int B, int H, int n, fl
     }
     const int T = row_tiles(n), np = sym_pairs(T), P = ctas_per_head(n);
     const int hp = sym_heads_per_pass(B, H, n);
-    const uint64_t cols = (uint64_t)H * D, npad = (uint64_t)T * TILE;
+    const uint64_t cols = (uint64_t)H * D;
     SymMaps maps;
-    if (!make_tensor_map_bf16_3d(&maps.x, X, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.o, out, B, n, cols, 128) ||
-        !make_tensor_map_f32(&maps.s, S, (uint64_t)hp * npad, npad, 128, 32))
+    if (!make_tensor_map_bf16_3d(&maps.x, X, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.o, out, B, n, cols, 128))
         return PSA_ERR_CUDA;
     for (int bh0 = 0; bh0 < B * H; bh0 += hp) {
         const int heads = min(hp, B * H - bh0);
-        sym_scores_kernel<D><<<heads * np, 128, Cfg::SCORES_SMEM, stream>>>(maps, n, H, bh0, scale, dc);
+        sym_scores_kernel<D><<<heads * np, 128, Cfg::SCORES_SMEM, stream>>>(maps, S, n, H, bh0, scale, dc);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) { set_cuda_error(e, "sym_scores_kernel launch"); return PSA_ERR_CUDA; }
-        sym_attn_kernel<D><<<heads * P, ATTN_THREADS, Cfg::SMEM, stream>>>(maps, n, H, bh0, heads, dc);
+        sym_attn_kernel<D><<<heads * P, ATTN_THREADS, Cfg::SMEM, stream>>>(maps, S, n, H, bh0, heads, dc);
         e = cudaGetLastError();
         if (e != cudaSuccess) { set_cuda_error(e, "sym_attn_kernel launch"); return PSA_ERR_CUDA; }
     }
@@ -452,8 +465,7 @@ int launch_symmetric(const void* X, void* out, float* S, int B, int H, int n, fl
 }  // namespace
 
 size_t bf16_symmetric_scratch_bytes(int B, int H, int n) {
-    const size_t npad = (size_t)row_tiles(n) * TILE;
-    return (size_t)sym_heads_per_pass(B, H, n) * npad * npad * sizeof(float);
+    return (size_t)sym_heads_per_pass(B, H, n) * sym_pairs(row_tiles(n)) * S_BLOCK_BYTES;
 }
 
 int bf16_attention(const void* Q, const void* K, const void* V, void* out, float* S, size_t s_bytes, int B, int H,

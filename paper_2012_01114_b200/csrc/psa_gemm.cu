@@ -77,25 +77,6 @@ bool make_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t batch,
     return true;
 }
 
-bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
-                         uint32_t box_cols) {
-    if (!resolve_encode()) return false;
-    cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 4};
-    cuuint32_t box[2] = {box_cols, box_rows};
-    cuuint32_t es[2] = {1, 1};
-    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-        char msg[96];
-        snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled (fp32) failed with CUresult %d", (int)r);
-        set_error_text(msg);
-        return false;
-    }
-    return true;
-}
-
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;

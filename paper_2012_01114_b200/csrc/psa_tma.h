@@ -18,9 +18,4 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uin
 bool make_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t batch, uint64_t n, uint64_t cols,
                              uint32_t box_rows);
 
-// Tensor map over a row-major [rows x cols] fp32 matrix (dense): boxes are [box_rows x box_cols] with
-// box_cols * 4 == 128 bytes, 128-byte swizzle.
-bool make_tensor_map_f32(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
-                         uint32_t box_cols);
-
 }  // namespace psa
