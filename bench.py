@@ -38,21 +38,28 @@ L2_FLUSH_BYTES = 256 << 20
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
-# (attn_kernel_c4_masked_n8192_d128.txt, gemm_and_attn_c3_masked_n1024_d64.txt).  Each figure is tied to the
-# SHA-256 of the kernel source it was measured on; once that source changes the roofline reports traffic = null.
+# (attn_persist_kernel_c4_masked_n8192_d128.txt, gemm_and_attn_persist_c3_masked_n1024_d64.txt).  Each figure is tied
+# to the SHA-256 of the sources of the kernel it was measured on; once one of them changes the roofline reports
+# traffic = null.
 NCU_TRAFFIC = {
     "sources": {
-        "attn": "fc68ce3e412a2c975dab5b3bbdf04c41081304e49a19d22d2f6693d69ddf062a",
-        "proj": "a0e3018c778ef73c0e369cb34617797055238c0b7013d90d881b6e8f2572c6cf",
-        "common": "f4c4c8e46254e54a9901d3bf7409741f97e645a86bd07fcca32545538100330c"
+        "psa_attn_persist.cu": "4e73010d53a22cd27c5e5b52bf50966cfa39925a8625b4e812ca6ead664080fd",
+        "psa_softmax.cuh": "26f2313be7a89cb71d2b9775b66c60b246852e53657d64273966f4bc96385390",
+        "psa_sched.h": "b5ac1fe785a492b9f6cbf57155e9b395d50689c125643e41ed935483668e9840",
+        "psa_gemm.cu": "b22c311fb626b2d17c762c5787b025c56264053801012169b0812cbd08bd7fd4",
+        "sm100.cuh": "ce4521e9596e3d452fcd0532bc570d2a288593b7720b1c1c6ed2806253b5045f"
+    },
+    "kernel_sources": {
+        "attn": ["psa_attn_persist.cu", "psa_softmax.cuh", "psa_sched.h", "sm100.cuh"],
+        "proj": ["psa_gemm.cu", "sm100.cuh"]
     },
     "traffic_bytes": {
         "c4": {
-            "attn": 251813632
+            "attn": 327422720
         },
         "c3": {
-            "attn": 37849856,
-            "proj": 16195328
+            "attn": 37888256,
+            "proj": 16230144
         }
     }
 }
@@ -60,14 +67,13 @@ NCU_TRAFFIC = {
 
 def ncu_traffic(workload, kernel):
     import hashlib
-    files = {"attn": "psa_attn.cu", "proj": "psa_gemm.cu", "common": "sm100.cuh"}
     try:
-        for key in (kernel, "common"):
-            with open(os.path.join(ROOT, "paper_2012_01114_b200", "csrc", files[key]), "rb") as f:
-                if hashlib.sha256(f.read()).hexdigest() != NCU_TRAFFIC["sources"][key]:
+        for name in NCU_TRAFFIC["kernel_sources"][kernel]:
+            with open(os.path.join(ROOT, "paper_2012_01114_b200", "csrc", name), "rb") as f:
+                if hashlib.sha256(f.read()).hexdigest() != NCU_TRAFFIC["sources"][name]:
                     return None
         return NCU_TRAFFIC["traffic_bytes"].get(workload, {}).get(kernel)
-    except OSError:
+    except (OSError, KeyError):
         return None
 
 
@@ -418,7 +424,7 @@ def main():
     dominant = "attn" if kern["attn"] >= kern["proj"] else "proj"
     alg = fl["core"] if dominant == "attn" else fl["proj"]
     achieved = alg / (kern[dominant] * 1e-3) / 1e12 if kern[dominant] > 0 else None
-    roofline = {"bound": "tensor", "kernel": "attn_kernel (fused scores-softmax-weighted sum)" if dominant == "attn" else "gemm_bf16_kernel (projections)",
+    roofline = {"bound": "tensor", "kernel": ("sym_scores_kernel + sym_attn_kernel (symmetric scheme, all passes)" if sym else "attn_persist_kernel (fused scores-softmax-weighted sum)") if dominant == "attn" else "gemm_bf16_kernel (projections)",
                 "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": (achieved / peaks["bf16_tflops"]) if achieved else None, "peak_source": peaks["source"] + " burst bf16",
                 "traffic": ncu_traffic(args.workload, dominant), "traffic_unit": "bytes per launch (ncu)",
