@@ -30,7 +30,8 @@ cudaError_t f32_attention(const float* Q, const float* K, const float* V, float*
 // C[w][M, N] = A[M, K] * Bw[w][K, N], bf16 row-major, fp32 accumulation.  Returns a psa_status.
 int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int nW, int M, int K, int N,
                  DeviceCounters* dc, cudaStream_t stream);
-// Q, K, V, out: [B, n, H, d] bf16.  S: scratch for PSA_SYMMETRIC ([heads_per_pass, n, n] fp32).
+// Q, K, V, out: [B, n, H, d] bf16.  S: scratch for PSA_SYMMETRIC (bf16_symmetric_scratch_bytes:
+// one 64 KB fp32 image per score block at or below the block diagonal, for the heads of one pass).
 int bf16_attention(const void* Q, const void* K, const void* V, void* out, float* S, size_t s_bytes, int B,
                    int H, int n, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
 size_t bf16_symmetric_scratch_bytes(int B, int H, int n);
