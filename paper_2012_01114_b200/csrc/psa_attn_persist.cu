@@ -46,10 +46,12 @@ struct PCfg {
     static constexpr int TILE_BYTES = 128 * D * 2;      // one Q, K or V tile
     static constexpr int KSTAGES = D == 128 ? 2 : 4;
     static constexpr int VSTAGES = D == 128 ? 2 : 4;
-    // output staging buffers of 32 rows x D columns: one for each of an item's 8 units (d = 64), 3 that the units
-    // take in turn (d = 128, where shared memory has no room for more)
-    static constexpr int STAGE_BYTES = 32 * D * 2;
-    static constexpr int STAGE_BUFS = D == 64 ? 8 : 3;
+    // output staging buffers.  d = 64: a unit is the two warps that share 32 rows (32 rows x 64 columns), one buffer
+    // for each of an item's 8 units.  d = 128: a unit is one warp (its 32 rows x 64 columns), and the 16 units of an
+    // item take 6 buffers in turn (shared memory has no room for more)
+    static constexpr bool WARP_UNITS = D == 128;
+    static constexpr int STAGE_BYTES = 32 * 64 * 2;
+    static constexpr int STAGE_BUFS = D == 64 ? 8 : 6;
     static constexpr int SMEM = (2 + KSTAGES + VSTAGES) * TILE_BYTES + STAGE_BUFS * STAGE_BYTES + 1024;
     static constexpr bool SEP_P = D == 64;
     static constexpr int TMEM_S = 0, TMEM_P = 256, TMEM_O = SEP_P ? 384 : 256;
@@ -395,8 +397,8 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
             const CtaWork work = cta_work(idx, n, masked, nbh, group);
             if (t >= work.ntiles) {
                 // no rows for this slot in this item: its units' turns at the staging buffers are passed on
-                if (part == 0 && lane == 0) {
-                    const uint32_t unit = it * 8u + 4u * t + q;
+                if ((Cfg::WARP_UNITS || part == 0) && lane == 0) {
+                    const uint32_t unit = Cfg::WARP_UNITS ? it * 16u + 8u * t + 4u * part + q : it * 8u + 4u * t + q;
                     const uint32_t sbuf = unit % Cfg::STAGE_BUFS, suse = unit / Cfg::STAGE_BUFS;
                     if (count_wait(&stage_released[sbuf], suse, abortp)) stage_released[sbuf] = suse + 1;
                 }
@@ -499,13 +501,13 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
             if (TPR == 2) xch_sum[t][part][r] = l_run;
             ok = named_bar_all(ok, pair_bar, 32 * TPR);
             if (!ok) break;
-            // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row), bf16.  The two warps
-            // that share 32 rows write them into a staging buffer (32 rows x D columns) and one lane hands
-            // it to TMA.  Buffers are taken in the fixed order of the units (item, slot, lane quarter); a unit
-            // waits until the store of the unit that last used its buffer has read it.
+            // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row), bf16.  A unit (a warp, or
+            // the two warps that share 32 rows) writes its rows into a staging buffer and one lane hands it to
+            // TMA.  Buffers are taken in the fixed order of the units; a unit waits until the store of the unit
+            // that last used its buffer has read it.
             tc_fence_after();
             const float inv = 1.f / (TPR == 2 ? l_run + xch_sum[t][part ^ 1][r] : l_run);
-            const uint32_t unit = it * 8u + 4u * t + q;
+            const uint32_t unit = Cfg::WARP_UNITS ? it * 16u + 8u * t + 4u * part + q : it * 8u + 4u * t + q;
             const uint32_t sbuf = unit % Cfg::STAGE_BUFS, suse = unit / Cfg::STAGE_BUFS;
             uint8_t* stage = sStage + sbuf * Cfg::STAGE_BYTES;
             ok = count_wait(&stage_released[sbuf], suse, abortp);
@@ -516,7 +518,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                     uint32_t v[32];
                     tmem_ld32(tO + 32 * c, v);
                     tc_wait_ld();
-                    uint8_t* sub = stage + (col / 64) * 4096;       // [32 rows x 64 columns] sub-tiles, 128-byte swizzle
+                    uint8_t* sub = stage + (Cfg::WARP_UNITS ? 0 : (col / 64) * 4096);   // [32 rows x 64 columns] sub-tiles, 128-byte swizzle
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         uint4 o;
@@ -529,11 +531,16 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                 }
                 fence_async_smem();
             }
-            // (a pair that gave up carries that into the vote at the top of the next item)
-            ok = named_bar_all(ok, pair_bar, 32 * TPR);
-            if (ok && part == 0 && lane == 0) {
-                for (int u = 0; u < Cfg::SUB; ++u)
-                    tma_store_3d(&maps.o, stage + u * 4096, h * D + 64 * u, It * TILE + q * 32, b);
+            // (a warp or pair that gave up carries that into the vote at the top of the next item)
+            if (Cfg::WARP_UNITS) ok = __all_sync(0xffffffffu, ok);
+            else ok = named_bar_all(ok, pair_bar, 32 * TPR);
+            if (ok && (Cfg::WARP_UNITS || part == 0) && lane == 0) {
+                if (Cfg::WARP_UNITS) {
+                    tma_store_3d(&maps.o, stage, h * D + part * OPT, It * TILE + q * 32, b);
+                } else {
+                    for (int u = 0; u < Cfg::SUB; ++u)
+                        tma_store_3d(&maps.o, stage + u * 4096, h * D + 64 * u, It * TILE + q * 32, b);
+                }
                 tma_store_commit();
                 tma_store_wait_read();   // the buffer may be rewritten; the global writes complete on their own
                 __threadfence_block();
