@@ -43,7 +43,7 @@ L2_FLUSH_BYTES = 256 << 20
 # traffic = null.
 NCU_TRAFFIC = {
     "sources": {
-        "psa_attn_persist.cu": "4e73010d53a22cd27c5e5b52bf50966cfa39925a8625b4e812ca6ead664080fd",
+        "psa_attn_persist.cu": "19362a3ebdf8670bcce2b1906642817cd8d86ed89896647dc5d86e24a1e26bac",
         "psa_softmax.cuh": "26f2313be7a89cb71d2b9775b66c60b246852e53657d64273966f4bc96385390",
         "psa_sched.h": "b5ac1fe785a492b9f6cbf57155e9b395d50689c125643e41ed935483668e9840",
         "psa_gemm.cu": "b22c311fb626b2d17c762c5787b025c56264053801012169b0812cbd08bd7fd4",
@@ -55,11 +55,11 @@ NCU_TRAFFIC = {
     },
     "traffic_bytes": {
         "c4": {
-            "attn": 327422720
+            "attn": 332312576
         },
         "c3": {
-            "attn": 37888256,
-            "proj": 16230144
+            "attn": 37910528,
+            "proj": 16195584
         }
     }
 }
