@@ -7,7 +7,7 @@
 //   sym_scores_kernel   phase 1, one CTA per unordered pair of 128-row tiles {I, J}, J <= I: the block
 //                       S_IJ = scale * X_I X_J^T on the tensor core, written ONCE to the scratch.  Blocks
 //                       above the diagonal are neither computed nor stored.
-//   sym_attn_kernel     phases 2 and 3 per pair of row tiles: the row of blocks S_I,* is fetched into shared
+//   sym_attn_kernel     phases 2 and 3 per 128-row tile: the row of blocks S_I,* is fetched into shared
 //                       memory -- block (I, J) as stored for J <= I, block (J, I) read transposed for
 //                       J > I (the reuse) -- then softmax and O += P V as in the fused kernel of the other
 //                       schemes (two threads per row, P written to TMEM as bf16, V = X staged by TMA,
@@ -41,7 +41,7 @@ struct SymCfg {
     static constexpr int TILE_BYTES = 128 * D * 2;      // one X tile (bf16)
     static constexpr int VSTAGES = D == 128 ? 2 : 4;
     static constexpr int SMEM = 2 * S_BLOCK_BYTES + VSTAGES * TILE_BYTES + 1024;
-    static constexpr int TMEM_P = 0, TMEM_O = 128;      // P0 P1 (64 columns each: 128 keys as bf16 pairs) | O0 O1
+    static constexpr int TMEM_P = 0, TMEM_O = 64;       // P (64 columns: 128 keys as bf16 pairs) | O (D columns)
     static constexpr int SCORES_SMEM = (S_BLOCK_BYTES > 2 * TILE_BYTES ? S_BLOCK_BYTES : 2 * TILE_BYTES) + 1024;
 };
 
@@ -153,47 +153,50 @@ sym_scores_kernel(const __grid_constant__ SymMaps maps, float* __restrict__ Sg, 
     if (warp == 0) tmem_dealloc(tmem, 128);
 }
 
-// Phases 2 and 3 of the symmetric scheme for one pair of row tiles of one head: softmax over the stored scores
-// and O = P X.  576 threads: warp 0 = TMA producer (score blocks, X tiles), warp 1 = MMA issuer, warps 2-9 /
-// 10-17 = softmax and epilogue of row tile 0 / 1, two threads per row.
+// Phases 2 and 3 of the symmetric scheme for one 128-row tile of one head: softmax over the stored scores and
+// O = P X.  320 threads: warp 0 = producer (score blocks and X tiles, bulk / TMA copies), warp 1 = MMA issuer,
+// warps 2-9 = softmax and epilogue, two threads per row.  The kernel is bound by the arrival of its score blocks
+// (64 KB per 128 x 128 weights), so these are double-buffered: block j + 1 is in flight while block j is in the
+// softmax, and a buffer is released as soon as its scores are in registers.
+constexpr int SYM_THREADS = 32 * (CTRL_WARPS + SOFTMAX_WARPS_PER_TILE);   // 320
+
 template <int D>
-__global__ void __launch_bounds__(ATTN_THREADS, 1)
-sym_attn_kernel(const __grid_constant__ SymMaps maps, const float* __restrict__ Sg, int n, int H, int bh0, int nbh,
+__global__ void __launch_bounds__(SYM_THREADS, 1)
+sym_attn_kernel(const __grid_constant__ SymMaps maps, const float* __restrict__ Sg, int n, int H, int bh0,
                 DeviceCounters* dc) {
     using Cfg = SymCfg<D>;
     constexpr int VST = Cfg::VSTAGES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* sS = smem;                                  // one 64 KB score block per row tile
+    uint8_t* sS = smem;                                  // two 64 KB score blocks (stages)
     uint8_t* sV = smem + 2 * S_BLOCK_BYTES;              // VSTAGES tiles of X
     __shared__ SymBars bars;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
-    __shared__ float xch_max[2][2][2][128];   // [block parity][tile][column half][row]
-    __shared__ float xch_sum[2][2][128];      // [tile][column half][row]
+    __shared__ float xch_max[2][2][128];      // [block parity][column half][row]
+    __shared__ float xch_sum[2][128];         // [column half][row]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int T = row_tiles(n);
     const int np = sym_pairs(T);
-    const CtaWork work = cta_work(blockIdx.x, n, 0, nbh, 1);
-    const int hl = work.bh;                              // head inside this pass
+    const int hl = blockIdx.x / T;                       // head inside this pass
+    const int It = blockIdx.x - hl * T;                  // row tile
     const int bh = bh0 + hl;
     const int b = bh / H, h = bh - b * H;
     const int col0 = h * D;
-    const int last_t = work.ntiles - 1;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int t = 0; t < 2; ++t) {
-            mbar_init(&bars.s_full[t], 1);
-            mbar_init(&bars.s_free[t], 32 * SOFTMAX_WARPS_PER_TILE);
-            mbar_init(&bars.p_ready[t], 32 * SOFTMAX_WARPS_PER_TILE);
-            mbar_init(&bars.o_done[t], 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars.s_full[s], 1);
+            mbar_init(&bars.s_free[s], 32 * SOFTMAX_WARPS_PER_TILE);
         }
+        mbar_init(&bars.p_ready[0], 32 * SOFTMAX_WARPS_PER_TILE);
+        mbar_init(&bars.o_done[0], 1);
         for (int s = 0; s < 4; ++s) { mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], 1); }
         fence_mbar_init();
     }
-    if (warp == 1) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
+    if (warp == 1) { tmem_alloc(&tmem_base_s, 256); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -202,24 +205,21 @@ sym_attn_kernel(const __grid_constant__ SymMaps maps, const float* __restrict__ 
 
     if (warp == 0) {
         if (lane == 0) {
-            // ------------------------------------------------------------ TMA producer
-            int s_loads[2] = {0, 0}, v_loads = 0;
+            // ------------------------------------------------------------ producer
+            int s_loads = 0, v_loads = 0;
             bool ok = true;
             for (int j = 0; j < T && ok; ++j) {
-                for (int t = 0; t < work.ntiles && ok; ++t) {
-                    // the slot's buffer is free once its softmax threads have read block j - 1 for the last time
-                    if (j > 0) ok = mbar_wait(&bars.s_free[t], (j - 1) & 1, abortp);
-                    if (!ok) break;
-                    const int It = work.tile0 + t;
-                    const int bi = j <= It ? It : j, bj = j <= It ? j : It;      // stored block (row tile, column tile)
-                    mbar_arrive_expect_tx(&bars.s_full[t], S_BLOCK_BYTES);
-                    const float* src = Sg + ((size_t)hl * np + bi * (bi + 1) / 2 + bj) * (S_BLOCK_BYTES / 4);
-                    for (int u = 0; u < S_COPIES; ++u)      // several copies in flight move a block faster than one
-                        bulk_load_1d(sS + t * S_BLOCK_BYTES + u * (S_BLOCK_BYTES / S_COPIES), src + u * (S_BLOCK_BYTES / S_COPIES / 4),
-                                     S_BLOCK_BYTES / S_COPIES, &bars.s_full[t]);
-                    ++s_loads[t];
-                }
+                const int st = j & 1;
+                // a stage is free once the softmax threads have taken block j - 2 into registers
+                if (j >= 2) ok = mbar_wait(&bars.s_free[st], ((j >> 1) - 1) & 1, abortp);
                 if (!ok) break;
+                const int bi = j <= It ? It : j, bj = j <= It ? j : It;      // stored block (row tile, column tile)
+                const float* src = Sg + ((size_t)hl * np + bi * (bi + 1) / 2 + bj) * (S_BLOCK_BYTES / 4);
+                mbar_arrive_expect_tx(&bars.s_full[st], S_BLOCK_BYTES);
+                for (int u = 0; u < S_COPIES; ++u)      // several copies in flight move a block faster than one
+                    bulk_load_1d(sS + st * S_BLOCK_BYTES + u * (S_BLOCK_BYTES / S_COPIES), src + u * (S_BLOCK_BYTES / S_COPIES / 4),
+                                 S_BLOCK_BYTES / S_COPIES, &bars.s_full[st]);
+                ++s_loads;
                 const int s = j % VST;
                 if (j >= VST) ok = mbar_wait(&bars.v_empty[s], ((j / VST) - 1) & 1, abortp);
                 if (!ok) break;
@@ -229,40 +229,36 @@ sym_attn_kernel(const __grid_constant__ SymMaps maps, const float* __restrict__ 
                 ++v_loads;
             }
             if (*abortp) {  // let copies already issued land before shared memory is released
-                for (int t = 0; t < 2; ++t)
-                    if (s_loads[t] > 0) mbar_wait_drain(&bars.s_full[t], (s_loads[t] - 1) & 1);
+                for (int c = max(0, s_loads - 2); c < s_loads; ++c) mbar_wait_drain(&bars.s_full[c & 1], (c >> 1) & 1);
                 for (int c = max(0, v_loads - VST); c < v_loads; ++c) mbar_wait_drain(&bars.v_full[c % VST], (c / VST) & 1);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            // ------------------------------------------------------------ MMA issuer: O_t (+)= P_t X_j (phase 3, Eq. 3)
+            // ------------------------------------------------------------ MMA issuer: O (+)= P X_j (phase 3, Eq. 3)
             const uint32_t idescO = umma_idesc_bf16(128, D, UMMA_K_MAJOR, UMMA_MN_MAJOR);
             const uint32_t v_lo = umma_desc_lo_mnmajor(smem_u32(sV), 16384);
+            const uint32_t dO = tmem + Cfg::TMEM_O, aP = tmem + Cfg::TMEM_P;
             unsigned long long pv_blocks = 0;
             bool ok = true;
             for (int j = 0; j < T && ok; ++j) {
                 const int sv = j % VST;
-                ok = mbar_wait(&bars.v_full[sv], (j / VST) & 1, abortp);
-                for (int t = 0; t < work.ntiles && ok; ++t) {
-                    ok = mbar_wait(&bars.p_ready[t], j & 1, abortp);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t v = v_lo + sv * (Cfg::TILE_BYTES >> 4);
-                    const uint32_t dO = tmem + Cfg::TMEM_O + t * D, aP = tmem + Cfg::TMEM_P + t * 64;
-                    if (j == 0) {
+                ok = mbar_wait(&bars.v_full[sv], (j / VST) & 1, abortp) && mbar_wait(&bars.p_ready[0], j & 1, abortp);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t v = v_lo + sv * (Cfg::TILE_BYTES >> 4);
+                if (j == 0) {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk)
-                            umma_ts(dO, aP + kk * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, kk != 0);
-                    } else {
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(dO, aP + kk * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, kk != 0);
+                } else {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk)
-                            umma_ts(dO, aP + kk * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, 1);
-                    }
-                    ++pv_blocks;
-                    umma_commit(&bars.o_done[t]);
-                    if (t == last_t) umma_commit(&bars.v_empty[sv]);
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(dO, aP + kk * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, 1);
                 }
+                ++pv_blocks;
+                umma_commit(&bars.o_done[0]);
+                umma_commit(&bars.v_empty[sv]);
             }
             if (pv_blocks) {
                 atomicAdd(&dc->pv_macs, pv_blocks * (unsigned long long)TILE * TILE * D);
@@ -275,146 +271,141 @@ sym_attn_kernel(const __grid_constant__ SymMaps maps, const float* __restrict__ 
         constexpr int CPT = 128 / TPR, NCH = CPT / 32, OPT = D / TPR;
         constexpr float sl2 = LOG2E;                          // the stored scores carry the 1/sqrt(d) factor already
         const int sw = warp - CTRL_WARPS;
-        const int t = sw / SOFTMAX_WARPS_PER_TILE;              // row tile of this warp
-        const int part = (sw % SOFTMAX_WARPS_PER_TILE) >> 2;    // which share of the row's columns
-        if (t < work.ntiles) {
-            const int q = warp & 3;                             // TMEM lane quarter this warp may access
-            const int r = q * 32 + lane;                        // row inside the tile = TMEM lane
-            const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
-            const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off + part * OPT;
-            const uint32_t tP = tmem + Cfg::TMEM_P + t * 64 + lane_off;
-            const int It = work.tile0 + t;
-            const int pair_bar = 1 + t * 4 + q;                 // named barrier of the warps sharing rows
-            const int tile_bar = 9 + t;                         // named barrier of all softmax warps of the tile
-            const int col_base = part * CPT;
-            const uint8_t* sblock = sS + t * S_BLOCK_BYTES;
-            float m_run = -INFINITY, l_run = 0.f;
-            bool ok = true;
-            for (int j = 0; j < T; ++j) {
-                ok = mbar_wait(&bars.s_full[t], j & 1, abortp);
-                ok = __all_sync(0xffffffffu, ok);
-                // keys beyond the sequence (ragged last block) carry no weight; `cb` = last kept column
-                const int nvalid = min(TILE, n - j * TILE);
-                const bool ragged = nvalid < TILE;
-                const int cb = nvalid - 1;
-                float mx = -INFINITY;
-                // 32 of this thread's scores: from the block as stored (column tile j at or below the row tile), or
+        const int part = sw >> 2;                               // which share of the row's columns
+        const int q = warp & 3;                                 // TMEM lane quarter this warp may access
+        const int r = q * 32 + lane;                            // row inside the tile = TMEM lane
+        const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
+        const uint32_t tO = tmem + Cfg::TMEM_O + lane_off + part * OPT;
+        const uint32_t tP = tmem + Cfg::TMEM_P + lane_off;
+        const int pair_bar = 1 + q;                             // named barrier of the two warps sharing rows
+        const int tile_bar = 9;                                 // named barrier of all softmax warps
+        const int col_base = part * CPT;
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int j = 0; j < T; ++j) {
+            const uint8_t* sblock = sS + (j & 1) * S_BLOCK_BYTES;
+            ok = mbar_wait(&bars.s_full[j & 1], (j >> 1) & 1, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+            // keys beyond the sequence (ragged last block) carry no weight; `cb` = last kept column
+            const int nvalid = min(TILE, n - j * TILE);
+            const bool ragged = nvalid < TILE;
+            const int cb = nvalid - 1;
+            float mx = -INFINITY;
+            uint32_t sreg[NCH][32];
+            if (ok) {
+                // ---- this thread's 64 scores: from the block as stored (column tile j at or below the row tile), or
                 // from the mirror block (j, I) read down its columns (the reused half)
-                auto load32 = [&](int c, uint32_t (&v)[32]) {
-                    if (j <= It) {
+                if (j <= It) {
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
                         const uint8_t* sub = sblock + ((col_base >> 5) + c) * S_SUB_BYTES;
 #pragma unroll
                         for (int g = 0; g < 8; ++g) {
                             const float4 f = *reinterpret_cast<const float4*>(sub + swz128_offset(r, g));
-                            v[4 * g] = __float_as_uint(f.x); v[4 * g + 1] = __float_as_uint(f.y);
-                            v[4 * g + 2] = __float_as_uint(f.z); v[4 * g + 3] = __float_as_uint(f.w);
+                            sreg[c][4 * g] = __float_as_uint(f.x); sreg[c][4 * g + 1] = __float_as_uint(f.y);
+                            sreg[c][4 * g + 2] = __float_as_uint(f.z); sreg[c][4 * g + 3] = __float_as_uint(f.w);
                         }
-                    } else {
-                        const uint8_t* sub = sblock + q * S_SUB_BYTES + (lane & 3) * 4;   // rows of the mirror block = my columns
+                    }
+                } else {
+                    const uint8_t* sub = sblock + q * S_SUB_BYTES + (lane & 3) * 4;   // rows of the mirror block = my columns
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c)
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
-                            v[i] = *reinterpret_cast<const uint32_t*>(sub + swz128_offset(col_base + 32 * c + i, lane >> 2));
-                    }
-                };
-                if (ok) {
-                    // ---- pass 1: maximum of this thread's scores
+                            sreg[c][i] = *reinterpret_cast<const uint32_t*>(sub + swz128_offset(col_base + 32 * c + i, lane >> 2));
+                }
 #pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        uint32_t v[32];
-                        load32(c, v);
-                        mx = ragged ? max_chunk32<true>(v, col_base + 32 * c, cb, mx)
-                                    : max_chunk32<false>(v, col_base + 32 * c, r, mx);
-                    }
-                }
-                // the two threads of a row exchange their half-row maxima (and leave together if either gave up a wait)
-                xch_max[j & 1][t][part][r] = mx;
-                ok = named_bar_all(ok, pair_bar, 64);
-                if (!ok) { mbar_arrive(&bars.s_free[t]); break; }
-                mx = fmaxf(mx, xch_max[j & 1][t][part ^ 1][r]);
-                const float mx2 = mx * sl2;
-                float alpha = 1.f;
-                if (mx2 > m_run + RESCALE_THRESHOLD) {   // also taken on the first block (m_run = -inf)
-                    alpha = ex2_mufu(m_run - mx2);
-                    m_run = mx2;
-                }
-                // P and O are still in use by PV_{j-1} until its commit.  A wait given up here is not acted on
-                // before the next pair barrier, so that the two threads of a row stay together.
-                if (j > 0) {
-                    ok = mbar_wait(&bars.o_done[t], (j - 1) & 1, abortp);
-                    ok = __all_sync(0xffffffffu, ok);
-                    tc_fence_after();
-                }
-                // ---- pass 2: P = exp2(S * log2 e - m) as bf16 into TMEM
-                float rowsum = 0.f;
-                if (ok) {
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        uint32_t v[32], pk[16];
-                        load32(c, v);
-                        const int kc = col_base + 32 * c;            // first key column of the chunk
-                        rowsum += ragged ? exp_chunk32<0, true>(v, sl2, -m_run, kc, cb, pk)
-                                         : exp_chunk32<0, false>(v, sl2, -m_run, kc, r, pk);
-                        tmem_st16(tP + (kc >> 1), pk);
-                    }
-                }
-                // the scores have been read for the last time: the producer may fetch the slot's next block
-                mbar_arrive(&bars.s_free[t]);
-                l_run = fmaf(l_run, alpha, rowsum);
-                if (ok && j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8
-#pragma unroll
-                    for (int c = 0; c < OPT / 32; ++c) {
-                        uint32_t v[32];
-                        tmem_ld32(tO + 32 * c, v);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                        tmem_st32(tO + 32 * c, v);
-                    }
-                }
-                tc_wait_st();
-                tc_fence_before();
-                mbar_arrive(&bars.p_ready[t]);
+                for (int c = 0; c < NCH; ++c)
+                    mx = ragged ? max_chunk32<true>(sreg[c], col_base + 32 * c, cb, mx)
+                                : max_chunk32<false>(sreg[c], col_base + 32 * c, r, mx);
             }
-            if (ok) ok = mbar_wait(&bars.o_done[t], (T - 1) & 1, abortp);
-            xch_sum[t][part][r] = l_run;
-            if (named_bar_all(ok, tile_bar, 32 * SOFTMAX_WARPS_PER_TILE)) {
-                // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row); the slot's score
-                // buffer, which no load targets any more, stages the bf16 tile for the TMA store
+            // the scores are in registers: the stage may take block j + 2
+            mbar_arrive(&bars.s_free[j & 1]);
+            // the two threads of a row exchange their half-row maxima (and leave together if either gave up a wait)
+            xch_max[j & 1][part][r] = mx;
+            ok = named_bar_all(ok, pair_bar, 64);
+            if (!ok) break;
+            mx = fmaxf(mx, xch_max[j & 1][part ^ 1][r]);
+            const float mx2 = mx * sl2;
+            float alpha = 1.f;
+            if (mx2 > m_run + RESCALE_THRESHOLD) {   // also taken on the first block (m_run = -inf)
+                alpha = ex2_mufu(m_run - mx2);
+                m_run = mx2;
+            }
+            // P and O are still in use by PV_{j-1} until its commit.  A wait given up here is not acted on
+            // before the next pair barrier, so that the two threads of a row stay together.
+            if (j > 0) {
+                ok = mbar_wait(&bars.o_done[0], (j - 1) & 1, abortp);
+                ok = __all_sync(0xffffffffu, ok);
                 tc_fence_after();
-                const float inv = 1.f / (l_run + xch_sum[t][part ^ 1][r]);
-                uint8_t* stage = sS + t * S_BLOCK_BYTES;
+            }
+            // ---- P = exp2(S * log2 e - m) as bf16 into TMEM
+            float rowsum = 0.f;
+            if (ok) {
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    uint32_t pk[16];
+                    const int kc = col_base + 32 * c;            // first key column of the chunk
+                    rowsum += ragged ? exp_chunk32<0, true>(sreg[c], sl2, -m_run, kc, cb, pk)
+                                     : exp_chunk32<0, false>(sreg[c], sl2, -m_run, kc, r, pk);
+                    tmem_st16(tP + (kc >> 1), pk);
+                }
+            }
+            l_run = fmaf(l_run, alpha, rowsum);
+            if (ok && j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8
 #pragma unroll
                 for (int c = 0; c < OPT / 32; ++c) {
-                    const int col = part * OPT + 32 * c;       // first of 32 output columns handled here
                     uint32_t v[32];
                     tmem_ld32(tO + 32 * c, v);
                     tc_wait_ld();
-                    uint8_t* sub = stage + (col / 64) * 16384;
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint4 o;
-                        o.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]) * inv, __uint_as_float(v[g * 8 + 1]) * inv);
-                        o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]) * inv, __uint_as_float(v[g * 8 + 3]) * inv);
-                        o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]) * inv, __uint_as_float(v[g * 8 + 5]) * inv);
-                        o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]) * inv, __uint_as_float(v[g * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(sub + swz128_offset(r, (col % 64) / 8 + g)) = o;
-                    }
+                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                    tmem_st32(tO + 32 * c, v);
                 }
-                fence_async_smem();
-                named_bar_sync(tile_bar, 32 * SOFTMAX_WARPS_PER_TILE);
-                if (sw == t * SOFTMAX_WARPS_PER_TILE && lane == 0) {
-                    for (int u = 0; u < Cfg::SUB; ++u)
-                        tma_store_3d(&maps.o, stage + u * 16384, col0 + 64 * u, It * TILE, b);
-                    tma_store_commit();
-                    tma_store_wait_read();   // smem may be released; the writes complete on their own
+            }
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(&bars.p_ready[0]);
+        }
+        if (ok) ok = mbar_wait(&bars.o_done[0], (T - 1) & 1, abortp);
+        xch_sum[part][r] = l_run;
+        if (named_bar_all(ok, tile_bar, 32 * SOFTMAX_WARPS_PER_TILE)) {
+            // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row); the first score stage,
+            // which no copy targets any more, stages the bf16 tile for the TMA store
+            tc_fence_after();
+            const float inv = 1.f / (l_run + xch_sum[part ^ 1][r]);
+            uint8_t* stage = sS;
+#pragma unroll
+            for (int c = 0; c < OPT / 32; ++c) {
+                const int col = part * OPT + 32 * c;       // first of 32 output columns handled here
+                uint32_t v[32];
+                tmem_ld32(tO + 32 * c, v);
+                tc_wait_ld();
+                uint8_t* sub = stage + (col / 64) * 16384;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    uint4 o;
+                    o.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]) * inv, __uint_as_float(v[g * 8 + 1]) * inv);
+                    o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]) * inv, __uint_as_float(v[g * 8 + 3]) * inv);
+                    o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]) * inv, __uint_as_float(v[g * 8 + 5]) * inv);
+                    o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]) * inv, __uint_as_float(v[g * 8 + 7]) * inv);
+                    *reinterpret_cast<uint4*>(sub + swz128_offset(r, (col % 64) / 8 + g)) = o;
                 }
+            }
+            fence_async_smem();
+            named_bar_sync(tile_bar, 32 * SOFTMAX_WARPS_PER_TILE);
+            if (sw == 0 && lane == 0) {
+                for (int u = 0; u < Cfg::SUB; ++u)
+                    tma_store_3d(&maps.o, stage + u * 16384, col0 + 64 * u, It * TILE, b);
+                tma_store_commit();
+                tma_store_wait_read();   // smem may be released; the writes complete on their own
             }
         }
     }
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && abort_flag) atomicExch(&dc->status, (int)PSA_ERR_TIMEOUT);
-    if (warp == 1) tmem_dealloc(tmem, 512);
+    if (warp == 1) tmem_dealloc(tmem, 256);
 }
 
 // Heads per pass: as many as the scratch cap allows, in passes of equal size (the scratch is reused from pass
@@ -444,7 +435,7 @@ int launch_symmetric(const void* X, void* out, float* S, int B, int H, int n, fl
         if (e != cudaSuccess) { set_cuda_error(e, "cudaFuncSetAttribute(symmetric attention)"); return PSA_ERR_CUDA; }
         attr_set = true;
     }
-    const int T = row_tiles(n), np = sym_pairs(T), P = ctas_per_head(n);
+    const int T = row_tiles(n), np = sym_pairs(T);
     const int hp = sym_heads_per_pass(B, H, n);
     const uint64_t cols = (uint64_t)H * D;
     SymMaps maps;
@@ -455,7 +446,7 @@ int launch_symmetric(const void* X, void* out, float* S, int B, int H, int n, fl
         sym_scores_kernel<D><<<heads * np, 128, Cfg::SCORES_SMEM, stream>>>(maps, S, n, H, bh0, scale, dc);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) { set_cuda_error(e, "sym_scores_kernel launch"); return PSA_ERR_CUDA; }
-        sym_attn_kernel<D><<<heads * P, ATTN_THREADS, Cfg::SMEM, stream>>>(maps, S, n, H, bh0, heads, dc);
+        sym_attn_kernel<D><<<heads * T, SYM_THREADS, Cfg::SMEM, stream>>>(maps, S, n, H, bh0, dc);
         e = cudaGetLastError();
         if (e != cudaSuccess) { set_cuda_error(e, "sym_attn_kernel launch"); return PSA_ERR_CUDA; }
     }
