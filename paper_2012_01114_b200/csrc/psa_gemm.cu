@@ -5,7 +5,8 @@
 // launch).  Warp 0 streams operand tiles with TMA into a shared-memory ring, warp 1 issues tcgen05 MMAs
 // (A K-major, B in its natural row-major form = MN-major) into one of two 256-column TMEM accumulators,
 // warps 2-5 drain the other accumulator (TMEM -> registers -> bf16 -> swizzled shared memory -> TMA
-// store), so that a tile's epilogue runs under the next tile's main loop.
+// store, 64 columns at a time through two staging buffers so that the stores overlap the conversion),
+// so that a tile's epilogue runs under the next tile's main loop.
 #include <stdio.h>
 
 #include <mutex>
@@ -89,8 +90,7 @@ constexpr int A_BYTES = BM * BK * 2;           // 16 KB, K-major [128 x 64]
 constexpr int B_SUB_BYTES = BK * 64 * 2;       // 8 KB, one [64 k-rows x 64 n] sub-tile
 constexpr int B_BYTES = NSUB * B_SUB_BYTES;    // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES; // 48 KB
-constexpr int OUT_COLS = 128;                  // the epilogue moves a tile out in column halves
-constexpr int OUT_BYTES = BM * OUT_COLS * 2;   // 32 KB output staging (two swizzled [128 x 64] sub-tiles)
+constexpr int OUT_BYTES = 2 * BM * 64 * 2;      // 32 KB output staging: two swizzled [128 x 64] sub-tiles used in turn
 constexpr int GEMM_THREADS = 192;
 constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + OUT_BYTES + 1024;  // + slack for 1024-byte alignment
 constexpr int TMEM_COLS = 2 * BN;              // two accumulators
@@ -216,40 +216,42 @@ gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, int
             const TileCoord c = tile_coord(t, mt, nt);
             bool live = true;
 #pragma unroll 1
-            for (int hh = 0; hh < BN / OUT_COLS; ++hh) {
-                // uniform across the four warps; also orders the previous output store (warp 2 lane 0 waited
-                // for it to have read the staging buffer) before the writes below
+            for (int u = 0; u < NSUB; ++u) {
+                // The tile leaves in 64-column sub-tiles through two staging buffers used in turn: while the TMA store
+                // of one reads its buffer, the next sub-tile is converted into the other.
+                // This barrier is uniform across the four warps; it also orders the store that last used this buffer
+                // (warp 2 lane 0 waited for it to have read the buffer) before the writes below.
                 if (!named_bar_all(ok, 1, 128)) { live = false; break; }
                 tc_fence_after();
+                uint8_t* sub = stage_out + (u & 1) * 16384;
+                uint32_t r[2][32];
+                const uint32_t src = tmem + (static_cast<uint32_t>(q * 32) << 16) + buf * BN + u * 64;
+                tmem_ld32(src, r[0]);
+                tmem_ld32(src + 32, r[1]);
+                tc_wait_ld();
 #pragma unroll
-                for (int c0 = 0; c0 < OUT_COLS; c0 += 32) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem + (static_cast<uint32_t>(q * 32) << 16) + buf * BN + hh * OUT_COLS + c0, r);
-                    tc_wait_ld();
-                    uint8_t* sub = stage_out + (c0 / 64) * 16384;
+                for (int c0 = 0; c0 < 2; ++c0) {
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {  // four 16-byte chunks of 8 bf16
                         uint4 v;
-                        v.x = pack_bf16x2(__uint_as_float(r[g * 8 + 0]), __uint_as_float(r[g * 8 + 1]));
-                        v.y = pack_bf16x2(__uint_as_float(r[g * 8 + 2]), __uint_as_float(r[g * 8 + 3]));
-                        v.z = pack_bf16x2(__uint_as_float(r[g * 8 + 4]), __uint_as_float(r[g * 8 + 5]));
-                        v.w = pack_bf16x2(__uint_as_float(r[g * 8 + 6]), __uint_as_float(r[g * 8 + 7]));
-                        *reinterpret_cast<uint4*>(sub + swz128_offset(row, (c0 % 64) / 8 + g)) = v;
+                        v.x = pack_bf16x2(__uint_as_float(r[c0][g * 8 + 0]), __uint_as_float(r[c0][g * 8 + 1]));
+                        v.y = pack_bf16x2(__uint_as_float(r[c0][g * 8 + 2]), __uint_as_float(r[c0][g * 8 + 3]));
+                        v.z = pack_bf16x2(__uint_as_float(r[c0][g * 8 + 4]), __uint_as_float(r[c0][g * 8 + 5]));
+                        v.w = pack_bf16x2(__uint_as_float(r[c0][g * 8 + 6]), __uint_as_float(r[c0][g * 8 + 7]));
+                        *reinterpret_cast<uint4*>(sub + swz128_offset(row, c0 * 4 + g)) = v;
                     }
                 }
-                if (hh == BN / OUT_COLS - 1) {
+                if (u == NSUB - 1) {
                     tc_fence_before();
                     mbar_arrive(&acc_empty[buf]);      // the accumulator may be overwritten by tile i + 2
                 }
                 fence_async_smem();
                 named_bar_sync(2, 128);
                 if (warp == 2 && lane == 0) {
-                    for (int u = 0; u < OUT_COLS / 64; ++u) {
-                        const int col = c.n0 + hh * OUT_COLS + 64 * u;
-                        if (col < N) tma_store_2d(&maps.c[c.w], stage_out + u * 16384, col, c.m0);
-                    }
-                    tma_store_commit();
-                    tma_store_wait_read();             // the staging buffer may be rewritten
+                    const int col = c.n0 + 64 * u;
+                    if (col < N) tma_store_2d(&maps.c[c.w], sub, col, c.m0);
+                    tma_store_commit();                // (an empty group when the sub-tile lies beyond N)
+                    tma_store_wait_read_1();           // the OTHER buffer, stored one sub-tile ago, may be rewritten
                 }
             }
             if (!live) { ok = false; break; }
