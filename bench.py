@@ -46,8 +46,8 @@ NCU_TRAFFIC = {
         "psa_attn_persist.cu": "19362a3ebdf8670bcce2b1906642817cd8d86ed89896647dc5d86e24a1e26bac",
         "psa_softmax.cuh": "26f2313be7a89cb71d2b9775b66c60b246852e53657d64273966f4bc96385390",
         "psa_sched.h": "b5ac1fe785a492b9f6cbf57155e9b395d50689c125643e41ed935483668e9840",
-        "psa_gemm.cu": "b22c311fb626b2d17c762c5787b025c56264053801012169b0812cbd08bd7fd4",
-        "sm100.cuh": "ce4521e9596e3d452fcd0532bc570d2a288593b7720b1c1c6ed2806253b5045f"
+        "psa_gemm.cu": "40aee68e878f71b318a422d7780369c41d78cc0b25fab601b69724467f24b16e",
+        "sm100.cuh": "e7db1e3c78bf7631d027fac7c3a8e2b2db487890b77e0de145ba17783a9ac464"
     },
     "kernel_sources": {
         "attn": ["psa_attn_persist.cu", "psa_softmax.cuh", "psa_sched.h", "sm100.cuh"],
@@ -58,8 +58,8 @@ NCU_TRAFFIC = {
             "attn": 332312576
         },
         "c3": {
-            "attn": 37910528,
-            "proj": 16195584
+            "attn": 37904384,
+            "proj": 16184320
         }
     }
 }
