@@ -55,7 +55,7 @@ NCU_TRAFFIC = {
     },
     "traffic_bytes": {
         "c4": {
-            "attn": 332312576
+            "attn": 329505280
         },
         "c3": {
             "attn": 37904384,
