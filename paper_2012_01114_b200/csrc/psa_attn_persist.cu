@@ -22,8 +22,9 @@
 // item: the next item's K, V and Q tiles are requested while the current item's last blocks are still
 // in the softmax, and its first scores are computed while the other row tile's output is written.
 //
-// CTA layout (576 threads): warp 0 = scheduler + TMA producer, warp 1 = MMA issuer, warps 2-9 = softmax
-// and epilogue of row tile 0, warps 10-17 = the same for row tile 1.  Within a tile's eight warps,
+// CTA layout (576 threads; 608 at d = 64): warp 0 = scheduler + TMA producer, warp 1 = MMA issuer, warps 2-9 =
+// softmax and epilogue of row tile 0, warps 10-17 = the same for row tile 1 (d = 64: warp 18 = MMA issuer of row
+// tile 1, warp 1 that of row tile 0).  Within a tile's eight warps,
 // warp pairs (w, w+4) share a TMEM lane quarter (32 rows) and split the 128 columns of S in halves;
 // the pair agrees on the row maximum through shared memory.
 // TMEM columns, d = 128: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_t (bf16, two per
@@ -84,10 +85,14 @@ __device__ __forceinline__ bool count_wait(const volatile uint32_t* counter, uin
     return true;
 }
 
-constexpr int ITEM_READERS = 1 + 2 * SOFTMAX_WARPS_PER_TILE;   // MMA issuer + one lane per softmax warp
+// d = 64 has an MMA-issuing thread per row tile slot (warp 1 for slot 0, the last warp for slot 1): a block there is
+// half the tensor work of d = 128 but as many instructions to issue, and one thread was measured to be the limit.
+constexpr int ISSUER1_WARP = CTRL_WARPS + 2 * SOFTMAX_WARPS_PER_TILE;
+template <int D> __host__ __device__ constexpr int persist_threads() { return ATTN_THREADS + (D == 64 ? 32 : 0); }
+template <int D> __host__ __device__ constexpr int item_readers() { return (D == 64 ? 2 : 1) + 2 * SOFTMAX_WARPS_PER_TILE; }   // issuers + one lane per softmax warp
 
 template <int D>
-__global__ void __launch_bounds__(ATTN_THREADS, 1)
+__global__ void __launch_bounds__(persist_threads<D>(), 1)
 attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme, int nbh,
                     int group, int nitems, float sl2, DeviceCounters* dc) {
     using Cfg = PCfg<D>;
@@ -116,7 +121,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
         for (int i = 0; i < 8; ++i) stage_released[i] = 0;
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bars.item_full[t], 1);
-            mbar_init(&bars.item_empty[t], ITEM_READERS);
+            mbar_init(&bars.item_empty[t], item_readers<D>());
             mbar_init(&bars.q_full[t], 1);
             mbar_init(&bars.q_empty[t], 1);
             mbar_init(&bars.s_full[t], 1);
@@ -125,8 +130,9 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
             mbar_init(&bars.o_done[t], 1);
         }
         for (int s = 0; s < 4; ++s) {
-            mbar_init(&bars.k_full[s], 1); mbar_init(&bars.k_empty[s], 1);
-            mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], 1);
+            // (with an issuer per slot, an operand tile collects one release from each of them)
+            mbar_init(&bars.k_full[s], 1); mbar_init(&bars.k_empty[s], SEP ? 2 : 1);
+            mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], SEP ? 2 : 1);
         }
         fence_mbar_init();
     }
@@ -204,17 +210,116 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                     mbar_wait_drain(&bars.v_full[c % VST], (c / VST) & 1);
             }
         }
+    } else if (SEP && (warp == 1 || warp == ISSUER1_WARP)) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ MMA issuer of row tile slot t (d = 64)
+            // The slot's blocks form a chain S_0, S_1 | PV_0, S_2 | PV_1, ...: with P in its own TMEM columns S_{j+1}
+            // needs only that the softmax warps have read S_j, PV_j needs P_j.  The thread issues the links in that
+            // order, sleeping on the barriers of each; the two slots' threads walk the item list independently.
+            const int t = warp == 1 ? 0 : 1;
+            const uint32_t idescS = umma_idesc_bf16(128, 128, UMMA_K_MAJOR, UMMA_K_MAJOR);
+            const uint32_t idescO = umma_idesc_bf16(128, D, UMMA_K_MAJOR, UMMA_MN_MAJOR);
+            unsigned long long qk_blocks = 0, pv_blocks = 0;
+            const uint32_t q_lo = umma_desc_lo_kmajor(smem_u32(sQ + t * Cfg::TILE_BYTES));
+            const uint32_t k_lo = umma_desc_lo_kmajor(smem_u32(sK));
+            const uint32_t v_lo = umma_desc_lo_mnmajor(smem_u32(sV), 16384);
+            const uint32_t dS = tmem + Cfg::TMEM_S + t * 128, dO = tmem + Cfg::TMEM_O + t * D;
+            const uint32_t aP = tmem + Cfg::TMEM_P + t * 64;
+            uint32_t kbase = 0, vbase = 0;      // ring positions of the current item's first K and V tile
+            uint32_t parts = 0;                 // earlier items in which this slot had rows
+            uint32_t blk0 = 0;                  // blocks of this slot in all earlier items
+            bool ok = true;
+            auto mma_S = [&](uint32_t kc) {     // S = Q K^T with K at ring position kc (phase 1, Eq. 1)
+                const uint32_t k = k_lo + (kc % KST) * (Cfg::TILE_BYTES >> 4);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = ((kk >> 2) * 16384 + (kk & 3) * 32) >> 4;
+                    umma_ss(dS, umma_desc_join(q_lo + off, UMMA_DESC_HI_SW128), umma_desc_join(k + off, UMMA_DESC_HI_SW128),
+                            idescS, kk != 0);
+                }
+                ++qk_blocks;
+            };
+            auto mma_PV = [&](uint32_t vc, bool first) {   // O (+)= P V with V at ring position vc (phase 3, Eq. 3)
+                const uint32_t v = v_lo + (vc % VST) * (Cfg::TILE_BYTES >> 4);
+                if (first) {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(dO, aP + kk * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, kk != 0);
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_ts(dO, aP + kk * 8, umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, 1);
+                }
+                ++pv_blocks;
+            };
+            // an operand tile has two releases to collect, one per slot; a slot whose partner has no block j gives both
+            auto release = [&](uint64_t* bar, bool both) {
+                umma_commit(bar);
+                if (both) umma_commit(bar);
+            };
+            for (uint32_t it = 0; ok; ++it) {
+                ok = mbar_wait(&bars.item_full[it & 1], (it >> 1) & 1, abortp);
+                if (!ok) break;
+                const int idx = item_ring[it & 1];
+                mbar_arrive(&bars.item_empty[it & 1]);
+                if (idx < 0) break;
+                const CtaWork work = cta_work(idx, n, masked, nbh, group);
+                const int nk0 = kv_tiles(work.tile0, T, scheme);
+                const int nk1 = work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0;
+                const int nkv = t ? nk1 : nk0, nkv_other = t ? nk0 : nk1;
+                if (nkv > 0) {
+                    // first scores of the item (the softmax warps must have taken the slot's previous scores out of TMEM)
+                    ok = mbar_wait(&bars.q_full[t], parts & 1, abortp) &&
+                         mbar_wait(&bars.k_full[kbase % KST], (kbase / KST) & 1, abortp);
+                    if (ok && blk0 > 0) ok = mbar_wait(&bars.s_free[t], (blk0 - 1) & 1, abortp);
+                    if (!ok) break;
+                    tc_fence_after();
+                    mma_S(kbase);
+                    umma_commit(&bars.s_full[t]);
+                    release(&bars.k_empty[kbase % KST], 0 >= nkv_other);
+                    if (nkv == 1) umma_commit(&bars.q_empty[t]);
+                    for (int j = 0; j < nkv && ok; ++j) {
+                        const uint32_t vc = vbase + j, kc = kbase + j + 1;
+                        if (j + 1 < nkv) {
+                            // S_{j+1} as soon as S_j has been read: it runs under the exponentials of block j
+                            ok = mbar_wait(&bars.k_full[kc % KST], (kc / KST) & 1, abortp) &&
+                                 mbar_wait(&bars.s_free[t], (blk0 + j) & 1, abortp);
+                            if (!ok) break;
+                            tc_fence_after();
+                            mma_S(kc);
+                            umma_commit(&bars.s_full[t]);
+                            release(&bars.k_empty[kc % KST], j + 1 >= nkv_other);
+                            if (j + 1 == nkv - 1) umma_commit(&bars.q_empty[t]);
+                        }
+                        ok = mbar_wait(&bars.v_full[vc % VST], (vc / VST) & 1, abortp) &&
+                             mbar_wait(&bars.p_ready[t], (blk0 + j) & 1, abortp);
+                        if (!ok) break;
+                        tc_fence_after();
+                        mma_PV(vc, j == 0);
+                        umma_commit(&bars.o_done[t]);
+                        release(&bars.v_empty[vc % VST], j >= nkv_other);
+                    }
+                    ++parts;
+                    blk0 += nkv;
+                }
+                kbase += max(nk0, nk1);
+                vbase += max(nk0, nk1);
+            }
+            const unsigned long long block_macs = (unsigned long long)TILE * TILE * D;
+            if (qk_blocks) atomicAdd(&dc->qk_macs, qk_blocks * block_macs);
+            if (pv_blocks) {
+                atomicAdd(&dc->pv_macs, pv_blocks * block_macs);
+                atomicAdd(&dc->exps, pv_blocks * (unsigned long long)(TILE * TILE));
+            }
+        }
     } else if (warp == 1) {
         if (lane == 0) {
             // ------------------------------------------------------------ MMA issuer
-            // Each row tile's blocks form a chain S_0, PV_0, S_1, PV_1, ...  The two tiles' chains are issued
+            // (d = 128) Each row tile's blocks form a chain S_0, PV_0, S_1, PV_1, ...  The two tiles' chains are issued
             // alternately: while the softmax warps of one tile work on their scores, the tensor pipe runs the
-            // other tile's MMAs, and it is this half-step offset that keeps the pipe busy.
-            //  * P over S (d = 128): PV_j and S_{j+1} of a tile go back to back under one commit, and the thread
-            //    sleeps on what each link needs, tile 0 then tile 1 then tile 0 ...
-            //  * P apart from S (d = 64): S_{j+1} needs only that S_j has been read, PV_j needs P_j; the two
-            //    tiles' events arrive in no fixed order, so the barriers are tested without blocking and
-            //    whatever has become possible is issued.
+            // other tile's MMAs, and it is this half-step offset that keeps the pipe busy.  P overlays S, so PV_j
+            // and S_{j+1} of a tile go back to back under one commit, and the thread sleeps on what each link
+            // needs, tile 0 then tile 1 then tile 0 ...
             const uint32_t idescS = umma_idesc_bf16(128, 128, UMMA_K_MAJOR, UMMA_K_MAJOR);
             const uint32_t idescO = umma_idesc_bf16(128, D, UMMA_K_MAJOR, UMMA_MN_MAJOR);
             unsigned long long qk_blocks = 0, pv_blocks = 0;
@@ -266,7 +371,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                 const int nkv[2] = {kv_tiles(work.tile0, T, scheme),
                                     work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0};
                 const int maxkv = max(nkv[0], nkv[1]);
-                if (!SEP) {
+                {
                     // first scores of both tiles
                     ok = mbar_wait(&bars.k_full[kbase % KST], (kbase / KST) & 1, abortp);
                     for (int t = 0; t < work.ntiles && ok; ++t) {
@@ -300,56 +405,6 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                                 if (t == work.ntiles - 1 || j + 1 >= nkv[t + 1]) umma_commit(&bars.k_empty[kc % KST]);
                                 if (j + 1 == nkv[t] - 1) umma_commit(&bars.q_empty[t]);
                             }
-                        }
-                    }
-                } else {
-                    int nS[2] = {0, 0}, nPV[2] = {0, 0};     // S and PV blocks issued for each tile in this item
-                    uint64_t t_last = 0;
-                    uint32_t idle = 0;
-                    // the K (V) tile at block j is released by whichever tile issues its S_j (PV_j) last
-                    auto k_last_user = [&](int t, int j) { const int o = t ^ 1; return j >= nkv[o] || nS[o] > j; };
-                    auto v_last_user = [&](int t, int j) { const int o = t ^ 1; return j >= nkv[o] || nPV[o] > j; };
-                    while (ok && (nPV[0] < nkv[0] || nPV[1] < nkv[1])) {
-                        bool progressed = false;
-                        for (int t = 0; t < work.ntiles; ++t) {
-                            int j = nS[t];
-                            if (j < nkv[t]) {
-                                const uint32_t kc = kbase + j, sidx = blk0[t] + j;
-                                bool rdy = mbar_test(&bars.k_full[kc % KST], (kc / KST) & 1);
-                                if (rdy && j == 0) rdy = mbar_test(&bars.q_full[t], parts[t] & 1);
-                                // the softmax warps must have taken the previous scores of this tile out of TMEM
-                                if (rdy && sidx > 0) rdy = mbar_test(&bars.s_free[t], (sidx - 1) & 1);
-                                if (rdy) {
-                                    tc_fence_after();
-                                    mma_S(t, kc);
-                                    umma_commit(&bars.s_full[t]);
-                                    ++nS[t];
-                                    if (k_last_user(t, j)) umma_commit(&bars.k_empty[kc % KST]);
-                                    if (j == nkv[t] - 1) umma_commit(&bars.q_empty[t]);
-                                    progressed = true;
-                                }
-                            }
-                            j = nPV[t];
-                            if (j < nkv[t] && j < nS[t]) {
-                                const uint32_t vc = vbase + j;
-                                bool rdy = mbar_test(&bars.p_ready[t], (blk0[t] + j) & 1);
-                                if (rdy) rdy = mbar_test(&bars.v_full[vc % VST], (vc / VST) & 1);
-                                if (rdy) {
-                                    tc_fence_after();
-                                    mma_PV(t, vc, j == 0);
-                                    umma_commit(&bars.o_done[t]);
-                                    ++nPV[t];
-                                    if (v_last_user(t, j)) umma_commit(&bars.v_empty[vc % VST]);
-                                    progressed = true;
-                                }
-                            }
-                        }
-                        if (progressed) {
-                            idle = 0;
-                        } else if ((++idle & 255u) == 0u) {
-                            if (*abortp) ok = false;
-                            else if (idle == 256u) t_last = globaltimer_ns();
-                            else if (globaltimer_ns() - t_last > 4 * PSA_WAIT_LIMIT_NS) { *abortp = 1; ok = false; }
                         }
                     }
                 }
@@ -580,7 +635,7 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
     const long long nitems = (long long)B * H * ctas_per_head(n);
     if (nitems > 0x7fffffffLL - sm_count) return PSA_ERR_SHAPE;
     const int grid = (int)(nitems < sm_count ? nitems : sm_count);
-    attn_persist_kernel<D><<<grid, ATTN_THREADS, Cfg::SMEM, stream>>>(
+    attn_persist_kernel<D><<<grid, persist_threads<D>(), Cfg::SMEM, stream>>>(
         maps, n, H, scheme, B * H, lpt_group(scheme, B * H, n, D), (int)nitems,
         scale * LOG2E, dc);
     const cudaError_t e = cudaGetLastError();
