@@ -24,13 +24,20 @@ struct Context {
     size_t own_bytes = 0;
     int own_device = -1;
     DeviceCounters* last_dc = nullptr;  // counters of the most recent call
+    // The workspace starts with two counter blocks.  The bf16 FULL / MASKED path uses them in turn: the attention
+    // kernel of a call clears the block of the next call, so that no clearing copy has to run ahead of the
+    // call's first kernel.  `clean_ws` is the workspace whose block `next_block` is known to be clear.
+    char* clean_ws = nullptr;
+    int next_block = 0;
     std::vector<cudaEvent_t> prof_events;  // 3 per profiled call
     int prof_calls = 0, prof_max = 0;
     psa_counts last_useful = {0, 0, 0, 0, 0, 0};
 };
 Context g_ctx;
 
-constexpr size_t COUNTER_BYTES = 256;
+constexpr size_t COUNTER_BYTES = 256;          // two counter blocks
+constexpr size_t COUNTER_BLOCK_BYTES = 128;
+static_assert(sizeof(DeviceCounters) <= COUNTER_BLOCK_BYTES, "counter block too small");
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -102,6 +109,7 @@ char* acquire_ws(size_t bytes) {
     e = cudaMalloc(&p, bytes);
     if (e != cudaSuccess) { set_cuda_error(e, "cudaMalloc(workspace)"); return nullptr; }
     g_ctx.own_ws = p;
+    g_ctx.clean_ws = nullptr;          // fresh memory: no counter block is known to be clear
     g_ctx.own_bytes = bytes;
     g_ctx.own_device = dev;
     return static_cast<char*>(p);
@@ -119,9 +127,18 @@ void useful_counts(int batch, int heads, int n, int d_model, int d_k, int scheme
 int run_layer(const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Q, const void* K,
               const void* V, int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, void* out,
               cudaStream_t stream, bool with_proj, char* ws, const WsLayout& L) {
-    DeviceCounters* dc = reinterpret_cast<DeviceCounters*>(ws);
-    cudaError_t e = cudaMemsetAsync(dc, 0, sizeof(DeviceCounters), stream);
-    if (e != cudaSuccess) { set_cuda_error(e, "cudaMemsetAsync(counters)"); return PSA_ERR_CUDA; }
+    const bool turns = dtype == PSA_BF16 && scheme != PSA_SYMMETRIC;   // the path whose last kernel clears the other block
+    int block = 0;
+    cudaError_t e = cudaSuccess;
+    if (turns && g_ctx.clean_ws == ws) {
+        block = g_ctx.next_block;
+    } else {
+        e = cudaMemsetAsync(ws, 0, 2 * COUNTER_BLOCK_BYTES, stream);
+        if (e != cudaSuccess) { set_cuda_error(e, "cudaMemsetAsync(counters)"); return PSA_ERR_CUDA; }
+    }
+    g_ctx.clean_ws = nullptr;           // until this call's kernels are known to be queued
+    DeviceCounters* dc = reinterpret_cast<DeviceCounters*>(ws + block * COUNTER_BLOCK_BYTES);
+    DeviceCounters* dc_next = turns ? reinterpret_cast<DeviceCounters*>(ws + (block ^ 1) * COUNTER_BLOCK_BYTES) : nullptr;
     g_ctx.last_dc = dc;
     memset(&g_ctx.last_useful, 0, sizeof(psa_counts));
     useful_counts(batch, heads, n, d_model, d_k, scheme, with_proj, &g_ctx.last_useful);
@@ -155,7 +172,12 @@ int run_layer(const void* X, const void* Wq, const void* Wk, const void* Wv, con
         if (e != cudaSuccess) { set_cuda_error(e, "f32_attention"); return PSA_ERR_CUDA; }
         return PSA_OK;
     }
-    return bf16_attention(Q, K, V, out, S, L.s_bytes, batch, heads, n, d_k, scale, scheme, dc, stream);
+    const int rc = bf16_attention(Q, K, V, out, S, L.s_bytes, batch, heads, n, d_k, scale, scheme, dc, dc_next, stream);
+    if (rc == PSA_OK && turns) {        // the other block will be clear once this call has run
+        g_ctx.clean_ws = ws;
+        g_ctx.next_block = block ^ 1;
+    }
+    return rc;
 }
 
 int layer_entry(const void* X, const void* Wq, const void* Wk, const void* Wv, int batch, int heads, int n,
@@ -329,6 +351,7 @@ int psa_set_workspace(void* dev_ptr, size_t bytes) {
     g_ctx.user_ws = dev_ptr;
     g_ctx.user_bytes = dev_ptr ? bytes : 0;
     g_ctx.last_dc = nullptr;
+    g_ctx.clean_ws = nullptr;
     return PSA_OK;
 }
 

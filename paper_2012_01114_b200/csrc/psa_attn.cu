@@ -460,8 +460,8 @@ size_t bf16_symmetric_scratch_bytes(int B, int H, int n) {
 }
 
 int bf16_attention(const void* Q, const void* K, const void* V, void* out, float* S, size_t s_bytes, int B, int H,
-                   int n, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream) {
-    if (scheme != PSA_SYMMETRIC) return bf16_attention_persist(Q, K, V, out, B, H, n, d, scale, scheme, dc, stream);
+                   int n, int d, float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream) {
+    if (scheme != PSA_SYMMETRIC) return bf16_attention_persist(Q, K, V, out, B, H, n, d, scale, scheme, dc, dc_next, stream);
     if (!S || s_bytes < bf16_symmetric_scratch_bytes(B, H, n)) return PSA_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(S) & 15u) != 0) return PSA_ERR_ALIGN;
     if (d == 64) return launch_symmetric<64>(Q, out, S, B, H, n, scale, dc, stream);

@@ -94,7 +94,7 @@ template <int D> __host__ __device__ constexpr int item_readers() { return (D ==
 template <int D>
 __global__ void __launch_bounds__(persist_threads<D>(), 1)
 attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme, int nbh,
-                    int group, int nitems, float sl2, DeviceCounters* dc) {
+                    int group, int nitems, float sl2, DeviceCounters* dc, DeviceCounters* dc_next) {
     using Cfg = PCfg<D>;
     constexpr bool SEP = Cfg::SEP_P;
     constexpr int KST = Cfg::KSTAGES, VST = Cfg::VSTAGES;
@@ -118,6 +118,8 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
+        // the counter block of the NEXT call on this workspace is cleared here, off that call's critical path
+        if (blockIdx.x == 0 && dc_next) *dc_next = DeviceCounters{0, 0, 0, 0, 0, 0};
         for (int i = 0; i < 8; ++i) stage_released[i] = 0;
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bars.item_full[t], 1);
@@ -615,7 +617,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
 
 template <int D>
 int launch_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, float scale,
-                   int scheme, DeviceCounters* dc, cudaStream_t stream) {
+                   int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream) {
     using Cfg = PCfg<D>;
     static bool attr_set = false;
     static int sm_count = 0;
@@ -637,7 +639,7 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
     const int grid = (int)(nitems < sm_count ? nitems : sm_count);
     attn_persist_kernel<D><<<grid, persist_threads<D>(), Cfg::SMEM, stream>>>(
         maps, n, H, scheme, B * H, lpt_group(scheme, B * H, n, D), (int)nitems,
-        scale * LOG2E, dc);
+        scale * LOG2E, dc, dc_next);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "attn_persist_kernel launch"); return PSA_ERR_CUDA; }
     return PSA_OK;
@@ -648,10 +650,10 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
 // FULL and MASKED schemes.  `dc->next_item` must be zero when the kernel starts (the per-call clearing of the
 // counter block does that); the kernel is launched once per call.
 int bf16_attention_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, int d,
-                           float scale, int scheme, DeviceCounters* dc, cudaStream_t stream) {
+                           float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream) {
     if (scheme != PSA_FULL && scheme != PSA_MASKED) return PSA_ERR_SCHEME_ARGS;
-    if (d == 64) return launch_persist<64>(Q, K, V, out, B, H, n, scale, scheme, dc, stream);
-    if (d == 128) return launch_persist<128>(Q, K, V, out, B, H, n, scale, scheme, dc, stream);
+    if (d == 64) return launch_persist<64>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
+    if (d == 128) return launch_persist<128>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
     return PSA_ERR_UNSUPPORTED;
 }
 

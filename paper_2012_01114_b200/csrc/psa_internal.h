@@ -32,12 +32,14 @@ int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int n
                  DeviceCounters* dc, cudaStream_t stream);
 // Q, K, V, out: [B, n, H, d] bf16.  S: scratch for PSA_SYMMETRIC (bf16_symmetric_scratch_bytes:
 // one 64 KB fp32 image per score block at or below the block diagonal, for the heads of one pass).
+// `dc_next`, if not null, is a second counter block that the call's attention kernel clears (FULL, MASKED only).
 int bf16_attention(const void* Q, const void* K, const void* V, void* out, float* S, size_t s_bytes, int B,
-                   int H, int n, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
+                   int H, int n, int d, float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next,
+                   cudaStream_t stream);
 size_t bf16_symmetric_scratch_bytes(int B, int H, int n);
 // The persistent fused kernel behind bf16_attention for PSA_FULL and PSA_MASKED (psa_attn_persist.cu).
 int bf16_attention_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, int d,
-                           float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
+                           float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream);
 
 void set_cuda_error(cudaError_t e, const char* where);
 void set_error_text(const char* text);

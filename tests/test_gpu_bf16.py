@@ -133,6 +133,28 @@ def test_reruns_are_bitwise_identical():
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
 
 
+def test_census_is_exact_in_any_sequence_of_calls():
+    # The FULL / MASKED path alternates between two counter blocks (the attention kernel of one call clears the block of
+    # the next); the other paths clear their block themselves.  Any interleaving must leave every call's census exact.
+    B, H, n, d = 2, 3, 384, 64
+    _, qb = inputs.tensor(5, 4, (B, n, H, d), 1.0, "bf16")
+    _, kb = inputs.tensor(5, 5, (B, n, H, d), 1.0, "bf16")
+    _, vb = inputs.tensor(5, 6, (B, n, H, d), 1.0, "bf16")
+    q, k, v = _dev_bf16(qb), _dev_bf16(kb), _dev_bf16(vb)
+    qf = q.float()
+    seq = [binding.MASKED, binding.MASKED, binding.FULL, binding.SYMMETRIC, binding.MASKED, "f32", binding.MASKED,
+           binding.FULL, binding.SYMMETRIC, binding.SYMMETRIC, binding.FULL]
+    for scheme in seq:
+        if scheme == "f32":
+            binding.psa_attention_core(qf, None, None, binding.SYMMETRIC)
+            st, got = binding.psa_last_issued()
+            assert st == binding.OK and got == binding.psa_skip_count(B, H, n, 0, d, binding.SYMMETRIC, binding.F32)
+            continue
+        args = (q, None, None) if scheme == binding.SYMMETRIC else (q, k, v)
+        binding.psa_attention_core(*args, scheme)
+        _check_census(B, H, n, 0, d, scheme)
+
+
 def test_host_entry_matches_device_entry():
     B, H, n, D, d = 1, 2, 256, 128, 64
     _, Xb = inputs.tensor(9, 0, (B, n, D), 1.0, "bf16")
