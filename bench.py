@@ -312,23 +312,30 @@ def main():
     H, scheme = w["heads"], w["scheme"]
     sym = scheme == psa.SYMMETRIC
 
-    def bf16_host(bits):
-        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+    f32 = w["dtype"] == "f32"            # workload c1: the fp32 CUDA-core path
+    tdtype = torch.float32 if f32 else torch.bfloat16
+    esize = 4 if f32 else 2
+
+    def bf16_host(arr):
+        if f32:
+            return torch.from_numpy(np.ascontiguousarray(arr, dtype=np.float32))
+        return torch.from_numpy(np.ascontiguousarray(arr).view(np.int16)).view(torch.bfloat16)
 
     if w["proj"]:
         host = {k: bf16_host(up[k]).pin_memory() for k in up}
         dev = {k: t.cuda() for k, t in host.items()}
-        out = torch.empty((w["batch"], w["n"], H * w["d_k"]), dtype=torch.bfloat16, device="cuda")
-        out_host = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+        out = torch.empty((w["batch"], w["n"], H * w["d_k"]), dtype=tdtype, device="cuda")
+        out_host = torch.empty(out.shape, dtype=tdtype).pin_memory()
+        layer = psa.psa_attention_f32 if f32 else psa.psa_attention
 
         def step():
-            psa.psa_attention(dev["X"], dev["Wq"], dev.get("Wk"), dev.get("Wv"), H, scheme, out=out)
+            layer(dev["X"], dev["Wq"], dev.get("Wk"), dev.get("Wv"), H, scheme, out=out)
         kernels_per_step = 2 + (1 if sym else 0)
     else:
         host = {k: bf16_host(up[k]).pin_memory() for k in up}
         dev = {k: t.cuda() for k, t in host.items()}
-        out = torch.empty((w["batch"], w["n"], H * w["d_k"]), dtype=torch.bfloat16, device="cuda")
-        out_host = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+        out = torch.empty((w["batch"], w["n"], H * w["d_k"]), dtype=tdtype, device="cuda")
+        out_host = torch.empty(out.shape, dtype=tdtype).pin_memory()
 
         def step():
             psa.psa_attention_core(dev["Q"], dev.get("K"), dev.get("V"), scheme, out=out)
@@ -395,7 +402,7 @@ def main():
         for _ in range(n_e2e):
             psa.psa_attention_host(host["X"], host["Wq"], host.get("Wk"), host.get("Wv"), H, scheme, out_host)
         e2e_s = time.perf_counter() - t0
-        h2d = sum(t.numel() * 2 for t in host.values())
+        h2d = sum(t.numel() * esize for t in host.values())
     else:
         n_e2e = min(args.steps, 10)
         e2e_stream = torch.cuda.current_stream()
@@ -412,13 +419,13 @@ def main():
         for _ in range(n_e2e):
             e2e_step()
         e2e_s = time.perf_counter() - t0
-        h2d = sum(t.numel() * 2 for t in host.values())
+        h2d = sum(t.numel() * esize for t in host.values())
     if world > 1:
         t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_s = float(t.item())
     e2e = None if args.no_e2e else {"value": aggregate([flops_step * n_e2e] * world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-           "d2h_bytes_per_step": int(out_host.numel() * 2), "steps": n_e2e,
+           "d2h_bytes_per_step": int(out_host.numel() * esize), "steps": n_e2e,
            "api": "psa_attention_host" if w["proj"] else "pinned copies + psa_attention_core"}
 
     if rank != 0:
@@ -439,13 +446,24 @@ def main():
                 "kernel_ms": kern, "kernel_ms_from": "in-library CUDA events around each kernel, second pass of the same steps",
                 "algorithmic_flops": alg,
                 "issued_flops": issued_flops}
+    if f32:
+        # The fp32 path runs on the CUDA cores and the 64-vector workload is a few microseconds of launch latency:
+        # its line reports the bytes it has to move against the measured copy bandwidth.
+        nbytes = 4.0 * sum(t.numel() for t in host.values()) + 4.0 * out.numel()
+        t_s = (kern["proj"] + kern["attn"]) * 1e-3
+        gbs = nbytes / t_s / 1e9 if t_s > 0 else None
+        roofline = {"bound": "hbm", "kernel": "f32_project_kernel + f32_attn_kernel (launch-latency bound at this size)",
+                    "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": (gbs / peaks["hbm_gbs"]) if gbs else None,
+                    "peak_source": peaks["source"] + " copy bandwidth", "traffic": None, "traffic_unit": "bytes per launch (ncu)",
+                    "kernel_ms": kern, "kernel_ms_from": "in-library CUDA events around each kernel, second pass of the same steps",
+                    "algorithmic_bytes": nbytes, "issued_flops": issued_flops}
     cpu = None
     if not args.no_cpu_baseline and world == 1:
         tf, cores, desc = oracle_sample(w)
         cpu = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": 1e3 * total_s / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic", "config": config_of(w, args), "clocks": clocks, "e2e": e2e,
+            "dtype": "f32" if f32 else "bf16", "data": "synthetic", "config": config_of(w, args), "clocks": clocks, "e2e": e2e,
             "gpu_launches": kernels_per_step * args.steps, "roofline": roofline, "cpu_baseline": cpu,
             "pct_of_measured_bf16_peak": 100.0 * value / world / peaks["bf16_tflops"],
             "pct_of_nominal_bf16_peak": 100.0 * value / world / 2250.0,
