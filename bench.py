@@ -43,7 +43,7 @@ L2_FLUSH_BYTES = 256 << 20
 # traffic = null.
 NCU_TRAFFIC = {
     "sources": {
-        "psa_attn_persist.cu": "679731613a140008ab34ddaa4d1d2b59898d0941728db8a2d7aa168379f92c90",
+        "psa_attn_persist.cu": "b28223940814d0e1cdef285b43bed2a14c502643deae604949d9ff56ea560333",
         "psa_softmax.cuh": "26f2313be7a89cb71d2b9775b66c60b246852e53657d64273966f4bc96385390",
         "psa_sched.h": "b5ac1fe785a492b9f6cbf57155e9b395d50689c125643e41ed935483668e9840",
         "psa_gemm.cu": "40aee68e878f71b318a422d7780369c41d78cc0b25fab601b69724467f24b16e",
@@ -55,11 +55,11 @@ NCU_TRAFFIC = {
     },
     "traffic_bytes": {
         "c4": {
-            "attn": 332348928
+            "attn": 329880576
         },
         "c3": {
-            "attn": 37856256,
-            "proj": 16212736
+            "attn": 37834240,
+            "proj": 16177152
         }
     }
 }
