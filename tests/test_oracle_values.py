@@ -211,6 +211,55 @@ def test_layer_splits_heads_by_column_blocks():
         assert cnt.mac1 == B * H * per_head
 
 
+def test_block_is_sum_over_heads_of_head_output_times_its_rows_of_wo():
+    # Output projection after the heads: z = sum_h y^(h) Wo[h*d:(h+1)*d, :], each y^(h) by library softmax/matmul.
+    rng = np.random.default_rng(5)
+    B, n, D, H, d = 2, 9, 6, 3, 4
+    X = rng.standard_normal((B, n, D)) * 0.5
+    Wq, Wk, Wv = (rng.standard_normal((D, H * d)) * 0.5 for _ in range(3))
+    Wo = rng.standard_normal((H * d, D)) * 0.5
+    for scheme in (oracle.FULL, oracle.MASKED, oracle.SYMMETRIC):
+        z, y, _ = oracle.attention_block(X, Wq, Wk, Wv, Wo, H, scheme)
+        assert z.shape == (B, n, D) and y.shape == (B, n, H * d)
+        for b in range(B):
+            want = np.zeros((n, D))
+            for h in range(H):
+                sl = slice(h * d, (h + 1) * d)
+                q = X[b] @ Wq[:, sl]
+                k = q if scheme == oracle.SYMMETRIC else X[b] @ Wk[:, sl]
+                v = q if scheme == oracle.SYMMETRIC else X[b] @ Wv[:, sl]
+                s = q @ k.T / math.sqrt(d)
+                if scheme == oracle.MASKED:
+                    s[np.triu_indices(n, 1)] = -np.inf
+                want += (scipy.special.softmax(s, axis=1) @ v) @ Wo[sl, :]
+            assert np.abs(z[b] - want).max() <= 1e-12
+
+
+def test_block_special_output_matrices():
+    rng = np.random.default_rng(6)
+    B, n, D, H, d = 1, 7, 8, 2, 4
+    X = rng.standard_normal((B, n, D)) * 0.5
+    Wq, Wk, Wv = (rng.standard_normal((D, H * d)) * 0.5 for _ in range(3))
+    y_ref, _ = oracle.attention_layer(X, Wq, Wk, Wv, H, oracle.MASKED)
+    # identity: the block is the layer
+    z, y, _ = oracle.attention_block(X, Wq, Wk, Wv, np.eye(H * d), H, oracle.MASKED)
+    assert np.array_equal(y, y_ref) and np.abs(z - y_ref).max() <= 1e-15
+    # a column selector picks one head's one component; zero gives zero
+    E = np.zeros((H * d, D)); E[5, 2] = 1.0
+    z, _, _ = oracle.attention_block(X, Wq, Wk, Wv, E, H, oracle.MASKED)
+    want = np.zeros((B, n, D)); want[..., 2] = y_ref[..., 5]
+    assert np.abs(z - want).max() <= 1e-15
+    # linear in Wo; not transposed (a non-square Wo would not even fit the other way round)
+    A = rng.standard_normal((H * d, 5)); Bm = rng.standard_normal((H * d, 5))
+    za, _, _ = oracle.attention_block(X, Wq, Wk, Wv, A, H, oracle.FULL)
+    zb, _, _ = oracle.attention_block(X, Wq, Wk, Wv, Bm, H, oracle.FULL)
+    zc, _, _ = oracle.attention_block(X, Wq, Wk, Wv, 2.0 * A - 3.0 * Bm, H, oracle.FULL)
+    assert za.shape == (B, n, 5) and np.abs(zc - (2.0 * za - 3.0 * zb)).max() <= 1e-12
+    # masked: the first output vector sees only the first value vector, z_0 = sum_h v_0^(h) Wo_h
+    zm, _, _ = oracle.attention_block(X, Wq, Wk, Wv, A, H, oracle.MASKED)
+    assert np.abs(zm[0, 0] - (X[0, 0] @ Wv) @ A).max() <= 1e-13
+
+
 def test_bf16_rounding_agrees_with_generator_and_torch():
     import torch
     rng = np.random.default_rng(5)
