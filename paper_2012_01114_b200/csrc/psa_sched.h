@@ -57,9 +57,16 @@ PSA_HD CtaWork cta_work(int cta, int n, int scheme_masked, int nbh, int group) {
 #ifndef PSA_LPT_MB
 #define PSA_LPT_MB 64
 #endif
+#ifndef PSA_LPT_ALL_FACTOR
+#define PSA_LPT_ALL_FACTOR 4
+#endif
 PSA_HD int lpt_group(int scheme, int nbh, int n, int d) {
     if (scheme != PSA_MASKED) return 1;
     const long long per_head = (long long)n * d * 2 * 2;
+    // (all heads in one group while their K and V together stay within about twice L2: CTAs that work on one head
+    // at the same time stream its key blocks in step, so the footprint at any moment is far below the total, and
+    // one longest-first list over everything balances best; measured on n = 8192 with 32 heads)
+    if (per_head * nbh <= ((long long)PSA_LPT_ALL_FACTOR * PSA_LPT_MB) << 20) return nbh;
     long long g = ((long long)PSA_LPT_MB << 20) / per_head;
     if (g < 1) g = 1;
     if (g > nbh) g = nbh;
