@@ -95,6 +95,8 @@ def useful_flops(w, batch=None):
     qk = d * (n * n if w["scheme"] == 0 else tri)
     pv = d * (tri if w["scheme"] == 2 else n * n)
     proj = ((1 if w["scheme"] == 1 else 3) * n * D * H * d) if w["proj"] else 0
+    if w.get("wo"):
+        proj += n * H * d * D            # output projection of the block workloads
     return {"core": 2.0 * B * H * (qk + pv), "proj": 2.0 * B * proj}
 
 
@@ -160,8 +162,12 @@ def oracle_sample(w, seconds_budget=20.0):
         done, t0 = 0, time.perf_counter()
         while True:
             b = done % w["batch"]
-            oracle.attention_layer(v["X"][b:b + 1], v["Wq"], v.get("Wk", v["Wq"]), v.get("Wv", v["Wq"]),
-                                   w["heads"], w["scheme"])
+            if w.get("wo"):
+                oracle.attention_block(v["X"][b:b + 1], v["Wq"], v.get("Wk", v["Wq"]), v.get("Wv", v["Wq"]), v["Wo"],
+                                       w["heads"], w["scheme"])
+            else:
+                oracle.attention_layer(v["X"][b:b + 1], v["Wq"], v.get("Wk", v["Wq"]), v.get("Wv", v["Wq"]),
+                                       w["heads"], w["scheme"])
             done += 1
             if time.perf_counter() - t0 > seconds_budget / 2:
                 break
@@ -206,6 +212,7 @@ def config_of(w, args):
     from paper_2012_01114_b200 import inputs
     return {"workload": w["name"], "batch": w["batch"], "heads": w["heads"], "n": w["n"], "d_model": w["d_model"] if w["proj"] else None,
             "d_k": w["d_k"], "scheme": inputs.SCHEME_NAMES[w["scheme"]], "projections": bool(w["proj"]),
+            "output_projection": bool(w.get("wo")),
             "parallelism": "replicas x%d (no exchange step)" % args.gpus,
             "l2": "flushed between steps by an untimed %d MiB memset" % (L2_FLUSH_BYTES >> 20)}
 
@@ -327,10 +334,16 @@ def main():
         out = torch.empty((w["batch"], w["n"], H * w["d_k"]), dtype=tdtype, device="cuda")
         out_host = torch.empty(out.shape, dtype=tdtype).pin_memory()
         layer = psa.psa_attention_f32 if f32 else psa.psa_attention
+        if w.get("wo"):
+            out = torch.empty((w["batch"], w["n"], w["d_model"]), dtype=tdtype, device="cuda")
+            out_host = torch.empty(out.shape, dtype=tdtype).pin_memory()
 
-        def step():
-            layer(dev["X"], dev["Wq"], dev.get("Wk"), dev.get("Wv"), H, scheme, out=out)
-        kernels_per_step = 2 + (1 if sym else 0)
+            def step():
+                psa.psa_attention_block(dev["X"], dev["Wq"], dev.get("Wk"), dev.get("Wv"), dev["Wo"], H, scheme, out=out)
+        else:
+            def step():
+                layer(dev["X"], dev["Wq"], dev.get("Wk"), dev.get("Wv"), H, scheme, out=out)
+        kernels_per_step = 2 + (1 if sym else 0) + (1 if w.get("wo") else 0)
     else:
         host = {k: bf16_host(up[k]).pin_memory() for k in up}
         dev = {k: t.cuda() for k, t in host.items()}
@@ -393,7 +406,7 @@ def main():
     e2e = None
     if args.no_e2e:
         n_e2e, e2e_s, h2d = 0, 1.0, 0
-    elif w["proj"]:
+    elif w["proj"] and not w.get("wo"):
         n_e2e = min(args.steps, 20)
         for _ in range(2):
             psa.psa_attention_host(host["X"], host["Wq"], host.get("Wk"), host.get("Wv"), H, scheme, out_host)
@@ -426,7 +439,8 @@ def main():
         e2e_s = float(t.item())
     e2e = None if args.no_e2e else {"value": aggregate([flops_step * n_e2e] * world, e2e_s), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": int(out_host.numel() * esize), "steps": n_e2e,
-           "api": "psa_attention_host" if w["proj"] else "pinned copies + psa_attention_core"}
+           "api": "pinned copies + psa_attention_block" if w.get("wo") else
+                  "psa_attention_host" if w["proj"] else "pinned copies + psa_attention_core"}
 
     if rank != 0:
         if world > 1:
@@ -437,7 +451,10 @@ def main():
     issued_flops = {"proj": 2.0 * issued["proj_macs"], "core": 2.0 * (issued["qk_macs"] + issued["pv_macs"])}
     kern = {"proj": proj_ms / max(calls, 1), "attn": attn_ms / max(calls, 1)}
     dominant = "attn" if kern["attn"] >= kern["proj"] else "proj"
-    alg = fl["core"] if dominant == "attn" else fl["proj"]
+    # (the in-library events bracket the input projections and the attention kernel; the output projection of the
+    # block workloads runs after them and is left out of the per-kernel figures)
+    wo_flops = 2.0 * w["batch"] * w["n"] * H * w["d_k"] * w["d_model"] if w.get("wo") else 0.0
+    alg = fl["core"] if dominant == "attn" else fl["proj"] - wo_flops
     achieved = alg / (kern[dominant] * 1e-3) / 1e12 if kern[dominant] > 0 else None
     roofline = {"bound": "tensor", "kernel": ("sym_scores_kernel + sym_attn_kernel (symmetric scheme, all passes)" if sym else "attn_persist_kernel (fused scores-softmax-weighted sum)") if dominant == "attn" else "gemm_bf16_kernel (projections)",
                 "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",

@@ -105,6 +105,26 @@ int psa_attention_host(const void* X_host, const void* Wq_host, const void* Wk_h
                        void* stream);
 
 /*
+ * Attention block: the layer above followed by the output projection over the concatenated heads,
+ *     z[b, i, :] = sum_h y^(h)[b, i, :] * Wo[h*d_k : (h+1)*d_k, :],
+ * y^(h) being the output of paper Eq. 3 for head h.  The paper's three phases end at y (Sec. 3.2) and it
+ * leaves the rest of the model to future work (Sec. 7); the multi-head remark of Sec. 3.1 implies that
+ * the heads' outputs are combined afterwards, and this is the usual way: one more product of the kind
+ * Sec. 3.1 calls a typical matrix-vector multiplication, run by the projection kernel.
+ *   X, Wq, Wk, Wv   as for psa_attention / psa_attention_f32 (dtype selects bf16 or fp32 storage).
+ *   Wo              device, [heads*d_k, d_model] row-major, same type; never NULL.
+ *   out             device, [batch, n, d_model] row-major, same type (caller-owned).
+ * y is kept in the workspace in the storage type (bf16 on the bf16 path) between the two steps; the
+ * workspace is psa_block_workspace_bytes(...).  No residual connection and no bias are added.
+ * After this call psa_last_issued reports proj_macs = input projections + batch*n*heads*d_k*d_model
+ * (the output projection); psa_skip_count describes the layer part only.
+ * Shape limits and errors as for psa_attention / psa_attention_f32; argument errors launch nothing.
+ */
+int psa_attention_block(const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Wo, int batch,
+                        int heads, int n, int d_model, int d_k, int scheme, int dtype, void* out, void* stream);
+size_t psa_block_workspace_bytes(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype);
+
+/*
  * Analytic census: what the tile scheduler will issue for this shape and scheme (paper Sec. 3.2,
  * 4.2, 5.2 for the useful_* fields).  Host only, launches nothing.  d_model = 0 means "core only"
  * (proj_macs = 0).

@@ -22,7 +22,8 @@ LIB_PATH = os.path.join(_HERE, "libpsa.so")
 
 EXPORTS = ("psa_attention", "psa_attention_f32", "psa_attention_core", "psa_attention_host", "psa_skip_count",
            "psa_last_issued", "psa_workspace_bytes", "psa_set_workspace", "psa_status_string",
-           "psa_last_cuda_error", "psa_profile_begin", "psa_profile_end", "psa_attention_sym_f32_noalloc")
+           "psa_last_cuda_error", "psa_profile_begin", "psa_profile_end", "psa_attention_sym_f32_noalloc",
+           "psa_attention_block", "psa_block_workspace_bytes")
 
 
 class PsaError(RuntimeError):
@@ -71,6 +72,10 @@ def lib() -> ctypes.CDLL:
         L.psa_profile_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
                                       ctypes.POINTER(ci)]
         L.psa_profile_end.restype = ci
+        L.psa_attention_block.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp]
+        L.psa_attention_block.restype = ci
+        L.psa_block_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ci, ci]
+        L.psa_block_workspace_bytes.restype = ctypes.c_size_t
         L.psa_attention_sym_f32_noalloc.argtypes = [vp, ci, ci, ci, ci, vp, vp]
         L.psa_attention_sym_f32_noalloc.restype = ci
         for f in ("psa_attention", "psa_attention_f32", "psa_attention_core", "psa_attention_host",
@@ -180,6 +185,30 @@ def psa_last_issued(stream=None):
     if rc not in (OK, ERR_TIMEOUT):
         raise PsaError(rc, "psa_last_issued")
     return rc, c.as_dict()
+
+
+def psa_attention_block(X, Wq, Wk, Wv, Wo, heads, scheme, out=None, stream=None):
+    """Projections + attention + output projection.  X [B,n,D], W* [D,heads*d_k], Wo [heads*d_k,D] -> out [B,n,D]
+    (all bf16 or all fp32, CUDA)."""
+    dtype = X.dtype
+    code = {torch.bfloat16: BF16, torch.float32: F32}[dtype]
+    for t, nm in ((X, "X"), (Wq, "Wq"), (Wk, "Wk"), (Wv, "Wv"), (Wo, "Wo"), (out, "out")):
+        _check_dev(t, dtype, nm)
+    batch, n, d_model = X.shape
+    hd = Wq.shape[1]
+    if Wq.shape[0] != d_model or hd % heads or Wo is None or tuple(Wo.shape) != (hd, d_model):
+        raise ValueError("Wq must be [d_model, heads*d_k] and Wo [heads*d_k, d_model]")
+    if out is None:
+        out = torch.empty((batch, n, d_model), dtype=dtype, device=X.device)
+    rc = lib().psa_attention_block(_ptr(X), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(Wo), batch, heads, n, d_model,
+                                   hd // heads, int(scheme), code, _ptr(out), _stream(stream))
+    if rc != OK:
+        raise PsaError(rc, "psa_attention_block")
+    return out
+
+
+def psa_block_workspace_bytes(batch, heads, n, d_model, d_k, scheme, dtype) -> int:
+    return int(lib().psa_block_workspace_bytes(batch, heads, n, d_model, d_k, int(scheme), int(dtype)))
 
 
 def psa_workspace_bytes(batch, heads, n, d_model, d_k, scheme, dtype, with_host_staging=False) -> int:

@@ -282,6 +282,50 @@ int psa_attention_host(const void* X_host, const void* Wq_host, const void* Wk_h
     return PSA_OK;
 }
 
+int psa_attention_block(const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Wo, int batch,
+                        int heads, int n, int d_model, int d_k, int scheme, int dtype, void* out, void* stream_v) {
+    g_err_text[0] = 0;
+    int rc = check_shape(batch, heads, n, d_model, d_k, scheme, dtype, true);
+    if (rc != PSA_OK) return rc;
+    if (!X || !Wq || !Wo || !out) return PSA_ERR_NULL;
+    if (scheme == PSA_SYMMETRIC) {
+        if ((Wk && Wk != Wq) || (Wv && Wv != Wq)) return PSA_ERR_SCHEME_ARGS;
+    } else if (!Wk || !Wv) {
+        return PSA_ERR_NULL;
+    }
+    if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(Wo) || !aligned16(out))
+        return PSA_ERR_ALIGN;
+    if (dtype == PSA_BF16 && (heads * d_k) % 64 != 0) return PSA_ERR_UNSUPPORTED;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    const WsLayout L = ws_layout(batch, heads, n, d_model, d_k, scheme, dtype, true, false);
+    const size_t y_off = align_up(L.total, 256);
+    const size_t y_bytes = (size_t)batch * n * heads * d_k * (dtype == PSA_BF16 ? 2 : 4);
+    char* ws = acquire_ws(y_off + align_up(y_bytes, 256));
+    if (!ws) return PSA_ERR_WORKSPACE;
+    void* y = ws + y_off;
+    rc = run_layer(X, Wq, Wk, Wv, nullptr, nullptr, nullptr, batch, heads, n, d_model, d_k, scheme, dtype, y, stream,
+                   true, ws, L);
+    if (rc != PSA_OK) return rc;
+    // z = y * Wo with the projection kernel; its MACs are added to the call's counter block
+    const void* Ws[3] = {Wo, Wo, Wo};
+    void* outs[3] = {out, out, out};
+    if (dtype == PSA_F32) {
+        cudaError_t e = f32_project(static_cast<const float*>(y), reinterpret_cast<const float* const*>(Ws),
+                                    reinterpret_cast<float* const*>(outs), 1, batch * n, heads * d_k, d_model,
+                                    g_ctx.last_dc, stream);
+        if (e != cudaSuccess) { set_cuda_error(e, "f32_project(Wo)"); return PSA_ERR_CUDA; }
+        return PSA_OK;
+    }
+    return bf16_project(y, Ws, outs, 1, batch * n, heads * d_k, d_model, g_ctx.last_dc, stream);
+}
+
+size_t psa_block_workspace_bytes(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype) {
+    if (d_model <= 0 || check_shape(batch, heads, n, d_model, d_k, scheme, dtype, true) != PSA_OK) return 0;
+    const WsLayout L = ws_layout(batch, heads, n, d_model, d_k, scheme, dtype, true, false);
+    return align_up(L.total, 256) + align_up((size_t)batch * n * heads * d_k * (dtype == PSA_BF16 ? 2 : 4), 256);
+}
+
 int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, psa_counts* c) {
     if (!c) return PSA_ERR_NULL;
     const bool with_proj = d_model > 0;

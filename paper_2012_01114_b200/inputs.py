@@ -109,6 +109,9 @@ WORKLOADS = {
     "c4": dict(batch=2, heads=16, n=8192, d_model=2048, d_k=128, dtype="bf16", scheme=MASKED, proj=False, seed=3,
                x_scale=1.0, w_scale=0.0),
 }
+# c2 / c3 followed by the output projection over the concatenated heads (Wo [heads*d_k, d_model], tensor id 7)
+for _b in ("c2", "c3"):
+    WORKLOADS[_b + "-block"] = dict(WORKLOADS[_b], wo=True, wo_scale=768 ** -0.5)
 for _n in (256, 1024, 4096, 16384):
     for _s in (FULL, SYMMETRIC, MASKED):
         WORKLOADS["c5-n%d-%s" % (_n, SCHEME_NAMES[_s])] = dict(
@@ -130,6 +133,8 @@ def make(name: str, batch: int | None = None, **override):
         ids = {"Wq": 1} if w["scheme"] == SYMMETRIC else {"Wq": 1, "Wk": 2, "Wv": 3}
         for k, t in ids.items():
             vals[k], up[k] = tensor(w["seed"], t, (D, H * d), w["w_scale"], w["dtype"])
+        if w.get("wo"):
+            vals["Wo"], up["Wo"] = tensor(w["seed"], 7, (H * d, D), w["wo_scale"], w["dtype"])
     else:
         ids = {"Q": 4} if w["scheme"] == SYMMETRIC else {"Q": 4, "K": 5, "V": 6}
         for k, t in ids.items():
