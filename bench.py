@@ -45,7 +45,7 @@ NCU_TRAFFIC = {
     "sources": {
         "psa_attn_persist.cu": "b28223940814d0e1cdef285b43bed2a14c502643deae604949d9ff56ea560333",
         "psa_softmax.cuh": "26f2313be7a89cb71d2b9775b66c60b246852e53657d64273966f4bc96385390",
-        "psa_sched.h": "b5ac1fe785a492b9f6cbf57155e9b395d50689c125643e41ed935483668e9840",
+        "psa_sched.h": "823e11ffb66560fea7e22933e754e6206902949b4ae780ebcdfaa400a541574d",
         "psa_gemm.cu": "40aee68e878f71b318a422d7780369c41d78cc0b25fab601b69724467f24b16e",
         "sm100.cuh": "e7db1e3c78bf7631d027fac7c3a8e2b2db487890b77e0de145ba17783a9ac464"
     },
@@ -55,11 +55,11 @@ NCU_TRAFFIC = {
     },
     "traffic_bytes": {
         "c4": {
-            "attn": 329880576
+            "attn": 592079872
         },
         "c3": {
-            "attn": 37834240,
-            "proj": 16177152
+            "attn": 37828096,
+            "proj": 16177408
         }
     }
 }

@@ -58,6 +58,24 @@ def test_projection_workloads_full(name):
     _census(w["batch"], w["heads"], w["n"], w["d_model"], w["d_k"], w["scheme"])
 
 
+@pytest.mark.parametrize("name", ["c2-block", "c3-block"])
+def test_block_workloads_full(name):
+    # the layer workloads followed by the output projection, every output element; tolerance of z: the layer's 2e-2
+    # plus the rounding of z itself to bf16 (at most 2^-8 |z|)
+    w = inputs.make(name)
+    v, u = w["values"], w["upload"]
+    out = binding.psa_attention_block(_dev_bf16(u["X"]), _dev_bf16(u["Wq"]), _dev_bf16(u["Wk"]), _dev_bf16(u["Wv"]),
+                                      _dev_bf16(u["Wo"]), w["heads"], w["scheme"])
+    ref, _, _ = oracle.attention_block(v["X"], v["Wq"], v["Wk"], v["Wv"], v["Wo"], w["heads"], w["scheme"])
+    excess = (np.abs(_f64(out) - ref) - 2.0 ** -8 * np.abs(ref)).max()
+    assert excess <= TOL_BF16, excess
+    st, got = binding.psa_last_issued()
+    B, H, n, D, d = w["batch"], w["heads"], w["n"], w["d_model"], w["d_k"]
+    assert st == binding.OK and got["proj_macs"] == 4 * B * n * D * H * d
+    t = oracle.tile_counts(n, d, w["scheme"], 128, 128)
+    assert got["qk_macs"] == B * H * t.issued_mac1 and got["pv_macs"] == B * H * t.issued_mac3
+
+
 def _edge_rows(n):
     rows = {0, 1, 63, 127, 128, 129, 255, 256, n // 2 - 1, n // 2, n - 257, n - 129, n - 128, n - 127, n - 2, n - 1}
     return sorted(r for r in rows if 0 <= r < n)
