@@ -463,6 +463,16 @@ def main():
                 "kernel_ms": kern, "kernel_ms_from": "in-library CUDA events around each kernel, second pass of the same steps",
                 "algorithmic_flops": alg,
                 "issued_flops": issued_flops}
+    if dominant == "attn" and kern["attn"] > 0 and not f32:
+        # Second ceiling of the attention kernel: one exponential per issued weight on the special-function pipe,
+        # 16 results per clock per SM (4 per scheduler), at the SM clock sampled during the timed region.
+        sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
+        xu_peak = 16.0 * sm_count * mhz * 1e6
+        xu_rate = issued["exps"] / (kern["attn"] * 1e-3)
+        roofline["second_ceiling"] = {"bound": "alu", "pipe": "MUFU ex2", "achieved": xu_rate / 1e12, "peak": xu_peak / 1e12,
+                                      "unit": "Texp/s", "frac": xu_rate / xu_peak,
+                                      "peak_from": "16 ex2 per clock per SM x %d SMs x %.0f MHz" % (sm_count, mhz)}
     if f32:
         # The fp32 path runs on the CUDA cores and the 64-vector workload is a few microseconds of launch latency:
         # its line reports the bytes it has to move against the measured copy bandwidth.
