@@ -340,7 +340,9 @@ int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme
         c->exps = c->useful_pv_macs / (uint64_t)d_k;
         return PSA_OK;
     }
-    // bf16: walk the CTA list and each CTA's block list exactly as the kernels do.
+    // bf16: walk the CTA list and each CTA's block list exactly as the kernels do.  (Where the kernel hands the last
+    // pairs of a launch out as single row tiles, split_point in psa_sched.h, those are the same row tiles with the
+    // same block lists taken one at a time: the census does not depend on the grouping.)
     const int T = row_tiles(n);
     const uint64_t block_macs = (uint64_t)TILE * TILE * d_k;
     uint64_t qk_blocks = 0, pv_blocks = 0;

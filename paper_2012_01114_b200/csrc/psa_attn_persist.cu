@@ -94,7 +94,7 @@ template <int D> __host__ __device__ constexpr int item_readers() { return (D ==
 template <int D>
 __global__ void __launch_bounds__(persist_threads<D>(), 1)
 attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme, int nbh,
-                    int group, int nitems, float sl2, DeviceCounters* dc, DeviceCounters* dc_next) {
+                    int group, int nitems, int split_arg, float sl2, DeviceCounters* dc, DeviceCounters* dc_next) {
     using Cfg = PCfg<D>;
     constexpr bool SEP = Cfg::SEP_P;
     constexpr int KST = Cfg::KSTAGES, VST = Cfg::VSTAGES;
@@ -115,6 +115,11 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int T = row_tiles(n);
     const int masked = scheme == PSA_MASKED;
+    // single-tile items at the end of the list exist at d = 64 only (a lone row tile gains nothing at d = 128)
+    auto item_work = [&](int idx) -> CtaWork {
+        if constexpr (D == 64) return cta_work_split(idx, n, masked, nbh, group, split_arg);
+        else return cta_work(idx, n, masked, nbh, group);
+    };
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -159,7 +164,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                 item_ring[slot] = idx < nitems ? idx : -1;
                 mbar_arrive(&bars.item_full[slot]);
                 if (idx >= nitems) break;
-                const CtaWork work = cta_work(idx, n, masked, nbh, group);
+                const CtaWork work = item_work(idx);
                 // the next item's index is fetched now, long before it is needed
                 const int next = (int)gridDim.x + (int)atomicAdd(&dc->next_item, 1u);
                 const int b = work.bh / H, h = work.bh - b * H;
@@ -265,7 +270,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                 const int idx = item_ring[it & 1];
                 mbar_arrive(&bars.item_empty[it & 1]);
                 if (idx < 0) break;
-                const CtaWork work = cta_work(idx, n, masked, nbh, group);
+                const CtaWork work = item_work(idx);
                 const int nk0 = kv_tiles(work.tile0, T, scheme);
                 const int nk1 = work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0;
                 const int nkv = t ? nk1 : nk0, nkv_other = t ? nk0 : nk1;
@@ -369,7 +374,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                 const int idx = item_ring[it & 1];
                 mbar_arrive(&bars.item_empty[it & 1]);
                 if (idx < 0) break;
-                const CtaWork work = cta_work(idx, n, masked, nbh, group);
+                const CtaWork work = item_work(idx);
                 const int nkv[2] = {kv_tiles(work.tile0, T, scheme),
                                     work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0};
                 const int maxkv = max(nkv[0], nkv[1]);
@@ -451,7 +456,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars.item_empty[it & 1]);
             if (idx < 0) break;
-            const CtaWork work = cta_work(idx, n, masked, nbh, group);
+            const CtaWork work = item_work(idx);
             if (t >= work.ntiles) {
                 // no rows for this slot in this item: its units' turns at the staging buffers are passed on
                 if ((Cfg::WARP_UNITS || part == 0) && lane == 0) {
@@ -634,12 +639,14 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
     if (!make_tensor_map_bf16_3d(&maps.q, Q, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.k, K, B, n, cols, 128) ||
         !make_tensor_map_bf16_3d(&maps.v, V, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.o, out, B, n, cols, 32))
         return PSA_ERR_CUDA;
-    const long long nitems = (long long)B * H * ctas_per_head(n);
+    const long long pairs = (long long)B * H * ctas_per_head(n);
+    const long long split = D == 64 ? split_point(scheme, pairs, n, sm_count) : pairs;
+    const long long nitems = pairs + (pairs - split);          // pairs, then the rest as single row tiles
     if (nitems > 0x7fffffffLL - sm_count) return PSA_ERR_SHAPE;
     const int grid = (int)(nitems < sm_count ? nitems : sm_count);
     attn_persist_kernel<D><<<grid, persist_threads<D>(), Cfg::SMEM, stream>>>(
         maps, n, H, scheme, B * H, lpt_group(scheme, B * H, n, D), (int)nitems,
-        scale * LOG2E, dc, dc_next);
+        split == pairs ? 0x7fffffff : (int)split, scale * LOG2E, dc, dc_next);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "attn_persist_kernel launch"); return PSA_ERR_CUDA; }
     return PSA_OK;

@@ -52,6 +52,25 @@ PSA_HD CtaWork cta_work(int cta, int n, int scheme_masked, int nbh, int group) {
     w.ntiles = left < TILES_PER_CTA ? left : TILES_PER_CTA;
     return w;
 }
+// The same list with a tail of single row tiles: items with an index at or beyond `split_from` are the two tiles of
+// pair split_from + (item - split_from) / 2, one item each (see split_point; every pair must have two tiles).
+PSA_HD CtaWork cta_work_split(int item, int n, int scheme_masked, int nbh, int group, int split_from) {
+    if (item < split_from) return cta_work(item, n, scheme_masked, nbh, group);
+    CtaWork w = cta_work(split_from + ((item - split_from) >> 1), n, scheme_masked, nbh, group);
+    w.tile0 += (item - split_from) & 1;
+    w.ntiles = 1;
+    return w;
+}
+// Work items of a launch over `pairs` pairs of row tiles on `sms` persistent CTAs: the first split_point() items are
+// pairs, the rest single row tiles.  Where all CTAs do the same work (FULL) and the last round of pairs would occupy
+// at most half of the CTAs, those pairs are handed out as single tiles instead, so that twice as many CTAs share
+// that round (a lone row tile takes less time than a pair at d_k = 64 and the same time at d_k = 128).
+PSA_HD long long split_point(int scheme, long long pairs, int n, int sms) {
+    if (scheme != PSA_FULL || (row_tiles(n) & 1) || sms <= 0) return pairs;
+    const long long r = pairs % sms;
+    if (r == 0 || 2 * r > sms) return pairs;
+    return pairs - r;
+}
 // Heads per group: as many as keep the group's K and V (bf16) within a fraction of L2; the schemes whose
 // CTAs all do the same work gain nothing from reordering and keep head-major order.
 #ifndef PSA_LPT_MB
