@@ -38,14 +38,15 @@ L2_FLUSH_BYTES = 256 << 20
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
-# (attn_persist_kernel_c4_masked_n8192_d128.txt, gemm_and_attn_persist_c3_masked_n1024_d64.txt).  Each figure is tied
+# (attn_persist_kernel_c4_masked_n8192_d128.txt, gemm_and_attn_persist_c3_masked_n1024_d64.txt,
+# attn_persist_kernel_c2_full_n512_d64.txt).  Each figure is tied
 # to the SHA-256 of the sources of the kernel it was measured on; once one of them changes the roofline reports
 # traffic = null.
 NCU_TRAFFIC = {
     "sources": {
-        "psa_attn_persist.cu": "b28223940814d0e1cdef285b43bed2a14c502643deae604949d9ff56ea560333",
+        "psa_attn_persist.cu": "48a23f568d24b9c64e89a6cbd36ec78b61d299df2155981757d1940d07cb5e1a",
         "psa_softmax.cuh": "26f2313be7a89cb71d2b9775b66c60b246852e53657d64273966f4bc96385390",
-        "psa_sched.h": "823e11ffb66560fea7e22933e754e6206902949b4ae780ebcdfaa400a541574d",
+        "psa_sched.h": "8bfeb6bc6f71007ef2d0044a38a0f5c4d9baf1f9cb73da7f6845232cda8598eb",
         "psa_gemm.cu": "40aee68e878f71b318a422d7780369c41d78cc0b25fab601b69724467f24b16e",
         "sm100.cuh": "e7db1e3c78bf7631d027fac7c3a8e2b2db487890b77e0de145ba17783a9ac464"
     },
@@ -55,11 +56,14 @@ NCU_TRAFFIC = {
     },
     "traffic_bytes": {
         "c4": {
-            "attn": 592079872
+            "attn": 596326912
         },
         "c3": {
-            "attn": 37828096,
-            "proj": 16177408
+            "attn": 37894400,
+            "proj": 16368896
+        },
+        "c2": {
+            "attn": 18940416
         }
     }
 }
