@@ -97,6 +97,8 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                     int group, int nitems, int split_arg, float sl2, DeviceCounters* dc, DeviceCounters* dc_next) {
     using Cfg = PCfg<D>;
     constexpr bool SEP = Cfg::SEP_P;
+    // (the experimental build with one softmax thread per row is kept working at d_k = 64 only)
+    static_assert(TPR == 2 || D == 64, "PSA_THREADS_PER_ROW=1 is not supported at d_k = 128");
     constexpr int KST = Cfg::KSTAGES, VST = Cfg::VSTAGES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));

@@ -14,7 +14,7 @@ namespace psa {
 #endif
 
 constexpr int CTRL_WARPS = 2;                       // producer, MMA issuer
-constexpr int TPR = PSA_THREADS_PER_ROW;            // softmax threads per query row (1 or 2)
+constexpr int TPR = PSA_THREADS_PER_ROW;            // softmax threads per query row: 2 (1 is an experiment, d_k = 64 only, slower)
 constexpr int SOFTMAX_WARPS_PER_TILE = 4 * TPR;
 constexpr int ATTN_THREADS = 32 * (CTRL_WARPS + 2 * SOFTMAX_WARPS_PER_TILE);   // 576
 constexpr float LOG2E = 1.4426950408889634f;
