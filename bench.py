@@ -44,8 +44,8 @@ L2_FLUSH_BYTES = 256 << 20
 # traffic = null.
 NCU_TRAFFIC = {
     "sources": {
-        "psa_attn_persist.cu": "48a23f568d24b9c64e89a6cbd36ec78b61d299df2155981757d1940d07cb5e1a",
-        "psa_softmax.cuh": "26f2313be7a89cb71d2b9775b66c60b246852e53657d64273966f4bc96385390",
+        "psa_attn_persist.cu": "ee15122883433bec99597dda82effe59e574edfea266f1fd984194237566eb60",
+        "psa_softmax.cuh": "083e8baadf062f616a29af748630250fe78a2611c588269cf94d2063a6550cac",
         "psa_sched.h": "8bfeb6bc6f71007ef2d0044a38a0f5c4d9baf1f9cb73da7f6845232cda8598eb",
         "psa_gemm.cu": "40aee68e878f71b318a422d7780369c41d78cc0b25fab601b69724467f24b16e",
         "sm100.cuh": "e7db1e3c78bf7631d027fac7c3a8e2b2db487890b77e0de145ba17783a9ac464"
@@ -56,14 +56,14 @@ NCU_TRAFFIC = {
     },
     "traffic_bytes": {
         "c4": {
-            "attn": 596326912
+            "attn": 592754176
         },
         "c3": {
-            "attn": 37894400,
-            "proj": 16368896
+            "attn": 37837824,
+            "proj": 16199936
         },
         "c2": {
-            "attn": 18940416
+            "attn": 18939904
         }
     }
 }
