@@ -105,6 +105,15 @@ int psa_attention_host(const void* X_host, const void* Wq_host, const void* Wk_h
                        void* stream);
 
 /*
+ * psa_attention_core with HOST buffers (paper Eq. 1-3 with q, k, v given): copies Q, K, V (one tensor for
+ * PSA_SYMMETRIC, where K_host and V_host are NULL or equal to Q_host) to staging buffers in the workspace,
+ * runs the core, copies `out` back to out_host and waits for `stream`.  Layouts, shape limits and errors as for
+ * psa_attention_core; pinned host memory makes the copies asynchronous up to the final wait.
+ */
+int psa_attention_core_host(const void* Q_host, const void* K_host, const void* V_host, int batch, int heads, int n,
+                            int d_k, int scheme, int dtype, void* out_host, void* stream);
+
+/*
  * Attention block: the layer above followed by the output projection over the concatenated heads,
  *     z[b, i, :] = sum_h y^(h)[b, i, :] * Wo[h*d_k : (h+1)*d_k, :],
  * y^(h) being the output of paper Eq. 3 for head h.  The paper's three phases end at y (Sec. 3.2) and it
@@ -137,6 +146,17 @@ int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme
  * device status (PSA_OK or PSA_ERR_TIMEOUT).
  */
 int psa_last_issued(void* stream, psa_counts* counts);
+
+/*
+ * Diagnostic of the bf16 path's online softmax (paper Eq. 2 evaluated block by block along the keys):
+ * waits for `stream`, then stores in *rescales how often, during the last call, a query row's running
+ * maximum was raised after the row's first key block -- each such event multiplies the row's partial
+ * output and partial row sum by exp(old maximum - new maximum).  The kernels raise the maximum only
+ * when it has grown by more than 2^8, so on inputs whose scores stay within a few units of each other
+ * the count is zero; it is nonzero when later keys carry much larger scores than earlier ones.
+ * The fp32 path finds each row's maximum before its first exponential and always reports zero.
+ */
+int psa_last_rescales(void* stream, uint64_t* rescales);
 
 /* Bytes of scratch memory a call with these arguments needs (projected q, k, v; the symmetric
  * scheme's score matrix; counters).  with_host_staging != 0 adds psa_attention_host's buffers. */
@@ -192,6 +212,35 @@ int psa_profile_end(float* proj_ms_sum, float* attn_ms_sum, int* calls);
 #define PSA_NOALLOC_MAX_SCORES (1u << 20)
 #define PSA_NOALLOC_SCRATCH_BYTES (256u + 4u * PSA_NOALLOC_MAX_SCORES)
 int psa_attention_sym_f32_noalloc(const void* X, int batch, int heads, int n, int d_k, void* out, void* stream);
+
+/*
+ * Measured rates of the SM pipes that phase 2 (paper Eq. 2) runs on, for the benchmark's second ceiling
+ * (the paper has no counterpart; it counts one exponent-accumulate per weight, Sec. 3.2).  Runs three short
+ * kernels on every SM (16 warps each, 8 independent instructions in flight per thread) and reports
+ * results per SM clock per SM, median over the SMs, best of three repetitions:
+ *   ex2_per_clk_per_sm               ex2.approx.ftz.f32 alone (the special-function unit)
+ *   fma_per_clk_per_sm               fma.rn.f32 alone
+ *   softmax_weights_per_clk_per_sm   the per-weight mix of the softmax's exponential pass:
+ *                                    fma (scale and shift), ex2, add (row sum), half a bf16x2 pack
+ * Synchronises `stream`; uses (and may grow) the workspace; psa_last_issued has nothing to report afterwards.
+ */
+typedef struct {
+    double ex2_per_clk_per_sm, fma_per_clk_per_sm, softmax_weights_per_clk_per_sm;
+    int sm_count;
+} psa_pipe_rates;
+int psa_measure_pipe_rates(psa_pipe_rates* rates, void* stream);
+
+/*
+ * Self-test of the failure path every kernel of the library shares (no counterpart in the paper).  All device-
+ * side waits are bounded; one that runs out raises a flag, the CTA's other waiters leave at their next poll,
+ * every role reaches the common teardown (tensor memory is freed) and PSA_ERR_TIMEOUT is written to the
+ * device status word.  A correct run never takes that path, so this call enqueues a one-CTA kernel built on
+ * the same skeleton whose barrier nobody completes, with a wait limit of `limit_us` microseconds
+ * (1 .. 100000).  It returns PSA_OK once the kernel is queued; the following psa_last_issued(stream, &c)
+ * must then return PSA_ERR_TIMEOUT with all counters zero, and later calls on the same context work as usual.
+ * Nothing traps or spins without a bound.
+ */
+int psa_selftest_wait_expiry(unsigned limit_us, void* stream);
 
 /* Text for a psa_status; never NULL. */
 const char* psa_status_string(int status);

@@ -23,7 +23,7 @@ LIB_PATH = os.path.join(_HERE, "libpsa.so")
 EXPORTS = ("psa_attention", "psa_attention_f32", "psa_attention_core", "psa_attention_host", "psa_skip_count",
            "psa_last_issued", "psa_workspace_bytes", "psa_set_workspace", "psa_status_string",
            "psa_last_cuda_error", "psa_profile_begin", "psa_profile_end", "psa_attention_sym_f32_noalloc",
-           "psa_attention_block", "psa_block_workspace_bytes")
+           "psa_attention_block", "psa_block_workspace_bytes", "psa_last_rescales", "psa_selftest_wait_expiry", "psa_measure_pipe_rates", "psa_attention_core_host")
 
 
 class PsaError(RuntimeError):
@@ -40,6 +40,11 @@ class Counts(ctypes.Structure):
 
     def as_dict(self):
         return {k: int(getattr(self, k)) for k, _ in self._fields_}
+
+
+class PipeRates(ctypes.Structure):
+    _fields_ = [("ex2_per_clk_per_sm", ctypes.c_double), ("fma_per_clk_per_sm", ctypes.c_double),
+                ("softmax_weights_per_clk_per_sm", ctypes.c_double), ("sm_count", ctypes.c_int)]
 
 
 _lib = None
@@ -76,6 +81,14 @@ def lib() -> ctypes.CDLL:
         L.psa_attention_block.restype = ci
         L.psa_block_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ci, ci]
         L.psa_block_workspace_bytes.restype = ctypes.c_size_t
+        L.psa_attention_core_host.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, vp]
+        L.psa_attention_core_host.restype = ci
+        L.psa_measure_pipe_rates.argtypes = [ctypes.POINTER(PipeRates), vp]
+        L.psa_measure_pipe_rates.restype = ci
+        L.psa_selftest_wait_expiry.argtypes = [ctypes.c_uint, vp]
+        L.psa_selftest_wait_expiry.restype = ci
+        L.psa_last_rescales.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
+        L.psa_last_rescales.restype = ci
         L.psa_attention_sym_f32_noalloc.argtypes = [vp, ci, ci, ci, ci, vp, vp]
         L.psa_attention_sym_f32_noalloc.restype = ci
         for f in ("psa_attention", "psa_attention_f32", "psa_attention_core", "psa_attention_host",
@@ -169,6 +182,22 @@ def psa_attention_host(X, Wq, Wk, Wv, heads, scheme, out, stream=None):
     return out
 
 
+def psa_attention_core_host(Q, K, V, scheme, out, stream=None):
+    """The attention core from HOST tensors Q, K, V [B,n,H,d] (CPU, contiguous; K = V = None for the symmetric
+    scheme) into the host tensor `out` [B,n,H*d]."""
+    dtype = Q.dtype
+    code = {torch.bfloat16: BF16, torch.float32: F32}[dtype]
+    for t in (Q, K, V, out):
+        if t is not None and (t.is_cuda or t.dtype != dtype or not t.is_contiguous()):
+            raise ValueError("host tensors must be contiguous CPU tensors of one dtype")
+    B, n, H, d = Q.shape
+    rc = lib().psa_attention_core_host(_ptr(Q), _ptr(K), _ptr(V), B, H, n, d, int(scheme), code, _ptr(out),
+                                       _stream(stream))
+    if rc != OK:
+        raise PsaError(rc, "psa_attention_core_host")
+    return out
+
+
 def psa_skip_count(batch, heads, n, d_model, d_k, scheme, dtype) -> dict:
     """Analytic census of what a call would issue (host only).  d_model = 0: core only."""
     c = Counts()
@@ -185,6 +214,31 @@ def psa_last_issued(stream=None):
     if rc not in (OK, ERR_TIMEOUT):
         raise PsaError(rc, "psa_last_issued")
     return rc, c.as_dict()
+
+
+def psa_measure_pipe_rates(stream=None) -> dict:
+    """Measured ex2 / fma / softmax-mix results per SM clock per SM (see include/psa.h)."""
+    r = PipeRates()
+    rc = lib().psa_measure_pipe_rates(ctypes.byref(r), _stream(stream))
+    if rc != OK:
+        raise PsaError(rc, "psa_measure_pipe_rates", "psa_attention_core_host")
+    return {k: getattr(r, k) for k, _ in r._fields_}
+
+
+def psa_selftest_wait_expiry(limit_us: int = 1000, stream=None):
+    """Queues the miniature kernel whose bounded wait expires; psa_last_issued() then reports ERR_TIMEOUT."""
+    rc = lib().psa_selftest_wait_expiry(int(limit_us), _stream(stream))
+    if rc != OK:
+        raise PsaError(rc, "psa_selftest_wait_expiry")
+
+
+def psa_last_rescales(stream=None) -> int:
+    """How often the last call raised a row's running softmax maximum after the row's first key block."""
+    v = ctypes.c_uint64()
+    rc = lib().psa_last_rescales(_stream(stream), ctypes.byref(v))
+    if rc != OK:
+        raise PsaError(rc, "psa_last_rescales", "psa_selftest_wait_expiry", "psa_measure_pipe_rates", "psa_attention_core_host")
+    return int(v.value)
 
 
 def psa_attention_block(X, Wq, Wk, Wv, Wo, heads, scheme, out=None, stream=None):

@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpsa.so")
-SOURCES = ["psa_api.cu", "psa_f32.cu", "psa_gemm.cu", "psa_attn.cu", "psa_attn_persist.cu", "psa_noalloc.cu"]
+SOURCES = ["psa_api.cu", "psa_f32.cu", "psa_gemm.cu", "psa_attn.cu", "psa_attn_persist.cu", "psa_noalloc.cu", "psa_selftest.cu", "psa_pipes.cu"]
 
 
 def _sources():
@@ -34,7 +34,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + ".%d.tmp" % os.getpid()
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-           "--use_fast_math" if False else "-DPSA_BUILD", "-Xcompiler", "-fPIC,-O2", "-shared", "-cudart", "static",
+           "-Xcompiler", "-fPIC,-O2", "-shared", "-cudart", "static",
            "-o", tmp] + os.environ.get("PSA_NVCC_FLAGS", "").split() + _sources()
     if verbose:
         cmd.insert(1, "-Xptxas=-v")

@@ -4,6 +4,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <mutex>
 #include <vector>
 
@@ -22,7 +23,6 @@ struct Context {
     size_t user_bytes = 0;
     void* own_ws = nullptr;
     size_t own_bytes = 0;
-    int own_device = -1;
     DeviceCounters* last_dc = nullptr;  // counters of the most recent call
     // The workspace starts with two counter blocks.  The bf16 FULL / MASKED path uses them in turn: the attention
     // kernel of a call clears the block of the next call, so that no clearing copy has to run ahead of the
@@ -33,7 +33,18 @@ struct Context {
     int prof_calls = 0, prof_max = 0;
     psa_counts last_useful = {0, 0, 0, 0, 0, 0};
 };
-Context g_ctx;
+// One context per device ordinal: workspace, counters and profiling state belong to the device that was current
+// when they were created.  Every entry point works on the context of the calling thread's current device.
+Context g_ctxs[MAX_DEVICES];
+std::mutex g_setup_mu;
+
+Context* current_ctx() {
+    int dev = 0;
+    const cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaGetDevice"); return nullptr; }
+    if (dev < 0 || dev >= MAX_DEVICES) { set_error_text("device ordinal beyond the library's table"); return nullptr; }
+    return &g_ctxs[dev];
+}
 
 constexpr size_t COUNTER_BYTES = 256;          // two counter blocks
 constexpr size_t COUNTER_BLOCK_BYTES = 128;
@@ -93,25 +104,21 @@ WsLayout ws_layout(int batch, int heads, int n, int d_model, int d_k, int scheme
 }
 
 // Returns the base of a workspace of at least `bytes`, or nullptr (error text set).
-char* acquire_ws(size_t bytes) {
-    if (g_ctx.user_ws && g_ctx.user_bytes >= bytes) return static_cast<char*>(g_ctx.user_ws);
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) { set_cuda_error(e, "cudaGetDevice"); return nullptr; }
-    if (g_ctx.own_ws && g_ctx.own_device == dev && g_ctx.own_bytes >= bytes) return static_cast<char*>(g_ctx.own_ws);
-    if (g_ctx.own_ws) {
+char* acquire_ws(Context& cx, size_t bytes) {
+    if (cx.user_ws && cx.user_bytes >= bytes) return static_cast<char*>(cx.user_ws);
+    if (cx.own_ws && cx.own_bytes >= bytes) return static_cast<char*>(cx.own_ws);
+    if (cx.own_ws) {
         cudaDeviceSynchronize();
-        cudaFree(g_ctx.own_ws);
-        g_ctx.own_ws = nullptr;
-        g_ctx.own_bytes = 0;
+        cudaFree(cx.own_ws);
+        cx.own_ws = nullptr;
+        cx.own_bytes = 0;
     }
     void* p = nullptr;
-    e = cudaMalloc(&p, bytes);
+    const cudaError_t e = cudaMalloc(&p, bytes);
     if (e != cudaSuccess) { set_cuda_error(e, "cudaMalloc(workspace)"); return nullptr; }
-    g_ctx.own_ws = p;
-    g_ctx.clean_ws = nullptr;          // fresh memory: no counter block is known to be clear
-    g_ctx.own_bytes = bytes;
-    g_ctx.own_device = dev;
+    cx.own_ws = p;
+    cx.clean_ws = nullptr;          // fresh memory: no counter block is known to be clear
+    cx.own_bytes = bytes;
     return static_cast<char*>(p);
 }
 
@@ -124,28 +131,28 @@ void useful_counts(int batch, int heads, int n, int d_model, int d_k, int scheme
     c->proj_macs = with_proj ? nproj * (uint64_t)batch * N * (uint64_t)d_model * (uint64_t)heads * d : 0;
 }
 
-int run_layer(const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Q, const void* K,
+int run_layer(Context& cx, const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Q, const void* K,
               const void* V, int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, void* out,
               cudaStream_t stream, bool with_proj, char* ws, const WsLayout& L) {
     const bool turns = dtype == PSA_BF16 && scheme != PSA_SYMMETRIC;   // the path whose last kernel clears the other block
     int block = 0;
     cudaError_t e = cudaSuccess;
-    if (turns && g_ctx.clean_ws == ws) {
-        block = g_ctx.next_block;
+    if (turns && cx.clean_ws == ws) {
+        block = cx.next_block;
     } else {
         e = cudaMemsetAsync(ws, 0, 2 * COUNTER_BLOCK_BYTES, stream);
         if (e != cudaSuccess) { set_cuda_error(e, "cudaMemsetAsync(counters)"); return PSA_ERR_CUDA; }
     }
-    g_ctx.clean_ws = nullptr;           // until this call's kernels are known to be queued
+    cx.clean_ws = nullptr;           // until this call's kernels are known to be queued
     DeviceCounters* dc = reinterpret_cast<DeviceCounters*>(ws + block * COUNTER_BLOCK_BYTES);
     DeviceCounters* dc_next = turns ? reinterpret_cast<DeviceCounters*>(ws + (block ^ 1) * COUNTER_BLOCK_BYTES) : nullptr;
-    g_ctx.last_dc = dc;
-    memset(&g_ctx.last_useful, 0, sizeof(psa_counts));
-    useful_counts(batch, heads, n, d_model, d_k, scheme, with_proj, &g_ctx.last_useful);
+    cx.last_dc = dc;
+    memset(&cx.last_useful, 0, sizeof(psa_counts));
+    useful_counts(batch, heads, n, d_model, d_k, scheme, with_proj, &cx.last_useful);
     const float scale = 1.0f / sqrtf((float)d_k);
     const int nW = scheme == PSA_SYMMETRIC ? 1 : 3;
     cudaEvent_t* pev = nullptr;
-    if (g_ctx.prof_calls < g_ctx.prof_max) pev = &g_ctx.prof_events[3 * g_ctx.prof_calls++];
+    if (cx.prof_calls < cx.prof_max) pev = &cx.prof_events[3 * cx.prof_calls++];
     struct EventTail {  // records the closing event on every exit path
         cudaEvent_t* ev; cudaStream_t st;
         ~EventTail() { if (ev) cudaEventRecord(ev[2], st); }
@@ -174,8 +181,8 @@ int run_layer(const void* X, const void* Wq, const void* Wk, const void* Wv, con
     }
     const int rc = bf16_attention(Q, K, V, out, S, L.s_bytes, batch, heads, n, d_k, scale, scheme, dc, dc_next, stream);
     if (rc == PSA_OK && turns) {        // the other block will be clear once this call has run
-        g_ctx.clean_ws = ws;
-        g_ctx.next_block = block ^ 1;
+        cx.clean_ws = ws;
+        cx.next_block = block ^ 1;
     }
     return rc;
 }
@@ -193,15 +200,34 @@ int layer_entry(const void* X, const void* Wq, const void* Wk, const void* Wv, i
     }
     if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(out)) return PSA_ERR_ALIGN;
     if (dtype == PSA_BF16 && (heads * d_k) % 64 != 0) return PSA_ERR_UNSUPPORTED;
-    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
     const WsLayout L = ws_layout(batch, heads, n, d_model, d_k, scheme, dtype, true, false);
-    char* ws = acquire_ws(L.total);
+    char* ws = acquire_ws(cx, L.total);
     if (!ws) return PSA_ERR_WORKSPACE;
-    return run_layer(X, Wq, Wk, Wv, nullptr, nullptr, nullptr, batch, heads, n, d_model, d_k, scheme, dtype, out,
+    return run_layer(cx, X, Wq, Wk, Wv, nullptr, nullptr, nullptr, batch, heads, n, d_model, d_k, scheme, dtype, out,
                      static_cast<cudaStream_t>(stream), true, ws, L);
 }
 
 }  // namespace
+
+int device_setup(DeviceSetup* st, cudaError_t (*configure)(), const char* what) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) { set_cuda_error(e, what); return 0; }
+    std::lock_guard<std::mutex> lock(g_setup_mu);
+    if (!st->done[dev]) {
+        int sms = 0;
+        e = configure();
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess || sms <= 0) { set_cuda_error(e, what); return 0; }
+        st->sm_count[dev] = sms;
+        st->done[dev] = true;
+    }
+    return st->sm_count[dev];
+}
 
 void set_cuda_error(cudaError_t e, const char* where) {
     snprintf(g_err_text, sizeof(g_err_text), "%s: %s", where, cudaGetErrorString(e));
@@ -237,11 +263,14 @@ int psa_attention_core(const void* Q, const void* K, const void* V, int batch, i
         return PSA_ERR_NULL;
     }
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(out)) return PSA_ERR_ALIGN;
-    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
     const WsLayout L = ws_layout(batch, heads, n, 0, d_k, scheme, dtype, false, false);
-    char* ws = acquire_ws(L.total);
+    char* ws = acquire_ws(cx, L.total);
     if (!ws) return PSA_ERR_WORKSPACE;
-    return run_layer(nullptr, nullptr, nullptr, nullptr, Q, K, V, batch, heads, n, 0, d_k, scheme, dtype, out,
+    return run_layer(cx, nullptr, nullptr, nullptr, nullptr, Q, K, V, batch, heads, n, 0, d_k, scheme, dtype, out,
                      static_cast<cudaStream_t>(stream), false, ws, L);
 }
 
@@ -259,9 +288,12 @@ int psa_attention_host(const void* X_host, const void* Wq_host, const void* Wk_h
     }
     if (dtype == PSA_BF16 && (heads * d_k) % 64 != 0) return PSA_ERR_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
     const WsLayout L = ws_layout(batch, heads, n, d_model, d_k, scheme, dtype, true, true);
-    char* ws = acquire_ws(L.total);
+    char* ws = acquire_ws(cx, L.total);
     if (!ws) return PSA_ERR_WORKSPACE;
     const size_t es = dtype == PSA_BF16 ? 2 : 4;
     const size_t xb = (size_t)batch * n * d_model * es, wb = (size_t)d_model * heads * d_k * es;
@@ -273,10 +305,49 @@ int psa_attention_host(const void* X_host, const void* Wq_host, const void* Wk_h
         if (e == cudaSuccess) e = cudaMemcpyAsync(ws + L.wv, Wv_host, wb, cudaMemcpyHostToDevice, stream);
     }
     if (e != cudaSuccess) { set_cuda_error(e, "cudaMemcpyAsync(H2D)"); return PSA_ERR_CUDA; }
-    rc = run_layer(ws + L.xs, ws + L.wq, ws + L.wk, ws + L.wv, nullptr, nullptr, nullptr, batch, heads, n, d_model,
+    rc = run_layer(cx, ws + L.xs, ws + L.wq, ws + L.wk, ws + L.wv, nullptr, nullptr, nullptr, batch, heads, n, d_model,
                    d_k, scheme, dtype, ws + L.outs, stream, true, ws, L);
     if (rc != PSA_OK) return rc;
     e = cudaMemcpyAsync(out_host, ws + L.outs, ob, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaMemcpyAsync(D2H)/sync"); return PSA_ERR_CUDA; }
+    return PSA_OK;
+}
+
+int psa_attention_core_host(const void* Q_host, const void* K_host, const void* V_host, int batch, int heads, int n,
+                            int d_k, int scheme, int dtype, void* out_host, void* stream_v) {
+    g_err_text[0] = 0;
+    int rc = check_shape(batch, heads, n, 0, d_k, scheme, dtype, false);
+    if (rc != PSA_OK) return rc;
+    if (!Q_host || !out_host) return PSA_ERR_NULL;
+    const bool sym = scheme == PSA_SYMMETRIC;
+    if (sym) {
+        if ((K_host && K_host != Q_host) || (V_host && V_host != Q_host)) return PSA_ERR_SCHEME_ARGS;
+    } else if (!K_host || !V_host) {
+        return PSA_ERR_NULL;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
+    const WsLayout L = ws_layout(batch, heads, n, 0, d_k, scheme, dtype, false, false);
+    const size_t tb = (size_t)batch * n * heads * d_k * (dtype == PSA_BF16 ? 2 : 4), tba = align_up(tb, 256);
+    const size_t q_off = align_up(L.total, 256), k_off = q_off + tba, v_off = k_off + tba;
+    const size_t o_off = sym ? k_off : v_off + tba;          // the symmetric scheme stages one input tensor
+    char* ws = acquire_ws(cx, o_off + tba);
+    if (!ws) return PSA_ERR_WORKSPACE;
+    cudaError_t e = cudaMemcpyAsync(ws + q_off, Q_host, tb, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess && !sym) {
+        e = cudaMemcpyAsync(ws + k_off, K_host, tb, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(ws + v_off, V_host, tb, cudaMemcpyHostToDevice, stream);
+    }
+    if (e != cudaSuccess) { set_cuda_error(e, "cudaMemcpyAsync(H2D)"); return PSA_ERR_CUDA; }
+    const void* q = ws + q_off;
+    rc = run_layer(cx, nullptr, nullptr, nullptr, nullptr, q, sym ? q : ws + k_off, sym ? q : ws + v_off, batch, heads, n,
+                   0, d_k, scheme, dtype, ws + o_off, stream, false, ws, L);
+    if (rc != PSA_OK) return rc;
+    e = cudaMemcpyAsync(out_host, ws + o_off, tb, cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) { set_cuda_error(e, "cudaMemcpyAsync(D2H)/sync"); return PSA_ERR_CUDA; }
     return PSA_OK;
@@ -297,14 +368,17 @@ int psa_attention_block(const void* X, const void* Wq, const void* Wk, const voi
         return PSA_ERR_ALIGN;
     if (dtype == PSA_BF16 && (heads * d_k) % 64 != 0) return PSA_ERR_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
     const WsLayout L = ws_layout(batch, heads, n, d_model, d_k, scheme, dtype, true, false);
     const size_t y_off = align_up(L.total, 256);
     const size_t y_bytes = (size_t)batch * n * heads * d_k * (dtype == PSA_BF16 ? 2 : 4);
-    char* ws = acquire_ws(y_off + align_up(y_bytes, 256));
+    char* ws = acquire_ws(cx, y_off + align_up(y_bytes, 256));
     if (!ws) return PSA_ERR_WORKSPACE;
     void* y = ws + y_off;
-    rc = run_layer(X, Wq, Wk, Wv, nullptr, nullptr, nullptr, batch, heads, n, d_model, d_k, scheme, dtype, y, stream,
+    rc = run_layer(cx, X, Wq, Wk, Wv, nullptr, nullptr, nullptr, batch, heads, n, d_model, d_k, scheme, dtype, y, stream,
                    true, ws, L);
     if (rc != PSA_OK) return rc;
     // z = y * Wo with the projection kernel; its MACs are added to the call's counter block
@@ -313,11 +387,11 @@ int psa_attention_block(const void* X, const void* Wq, const void* Wk, const voi
     if (dtype == PSA_F32) {
         cudaError_t e = f32_project(static_cast<const float*>(y), reinterpret_cast<const float* const*>(Ws),
                                     reinterpret_cast<float* const*>(outs), 1, batch * n, heads * d_k, d_model,
-                                    g_ctx.last_dc, stream);
+                                    cx.last_dc, stream);
         if (e != cudaSuccess) { set_cuda_error(e, "f32_project(Wo)"); return PSA_ERR_CUDA; }
         return PSA_OK;
     }
-    return bf16_project(y, Ws, outs, 1, batch * n, heads * d_k, d_model, g_ctx.last_dc, stream);
+    return bf16_project(y, Ws, outs, 1, batch * n, heads * d_k, d_model, cx.last_dc, stream);
 }
 
 size_t psa_block_workspace_bytes(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype) {
@@ -370,18 +444,95 @@ int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme
 
 int psa_last_issued(void* stream, psa_counts* c) {
     if (!c) return PSA_ERR_NULL;
-    std::lock_guard<std::mutex> lock(g_ctx.mu);
-    if (!g_ctx.last_dc) return PSA_ERR_NULL;
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
+    if (!cx.last_dc) return PSA_ERR_NULL;
     DeviceCounters h;
     cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
-    if (e == cudaSuccess) e = cudaMemcpy(&h, g_ctx.last_dc, sizeof(h), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(&h, cx.last_dc, sizeof(h), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) { set_cuda_error(e, "psa_last_issued"); return PSA_ERR_CUDA; }
-    *c = g_ctx.last_useful;
+    *c = cx.last_useful;
     c->proj_macs = h.proj_macs;
     c->qk_macs = h.qk_macs;
     c->pv_macs = h.pv_macs;
     c->exps = h.exps;
     return h.status;
+}
+
+int psa_measure_pipe_rates(psa_pipe_rates* r, void* stream_v) {
+    g_err_text[0] = 0;
+    if (!r) return PSA_ERR_NULL;
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess || sms <= 0) { set_cuda_error(e, "psa_measure_pipe_rates"); return PSA_ERR_CUDA; }
+    const size_t cyc_bytes = align_up(3 * (size_t)sms * sizeof(unsigned long long), 256);
+    char* ws = acquire_ws(cx, COUNTER_BYTES + cyc_bytes + 256);
+    if (!ws) return PSA_ERR_WORKSPACE;
+    cx.clean_ws = nullptr;
+    cx.last_dc = nullptr;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    unsigned long long* cyc = reinterpret_cast<unsigned long long*>(ws + COUNTER_BYTES);
+    std::vector<unsigned long long> h(3 * (size_t)sms);
+    double best[3] = {0, 0, 0};
+    for (int rep = 0; rep < 3; ++rep) {       // the first repetition warms the clocks up; the best is kept
+        e = cudaMemsetAsync(cyc, 0, cyc_bytes, stream);
+        if (e == cudaSuccess) e = launch_pipe_rates(cyc, reinterpret_cast<float*>(ws + COUNTER_BYTES + cyc_bytes), sms, stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+        if (e == cudaSuccess) e = cudaMemcpy(h.data(), cyc, h.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) { set_cuda_error(e, "psa_measure_pipe_rates"); return PSA_ERR_CUDA; }
+        for (int m = 0; m < 3; ++m) {
+            std::vector<unsigned long long> v(h.begin() + (size_t)m * sms, h.begin() + (size_t)(m + 1) * sms);
+            std::sort(v.begin(), v.end());
+            const double med = (double)v[v.size() / 2];
+            if (med > 0 && pipe_results_per_launch_per_sm() / med > best[m]) best[m] = pipe_results_per_launch_per_sm() / med;
+        }
+    }
+    r->ex2_per_clk_per_sm = best[0];
+    r->fma_per_clk_per_sm = best[1];
+    r->softmax_weights_per_clk_per_sm = best[2];
+    r->sm_count = sms;
+    return PSA_OK;
+}
+
+int psa_selftest_wait_expiry(unsigned limit_us, void* stream_v) {
+    g_err_text[0] = 0;
+    if (limit_us == 0 || limit_us > 100000u) return PSA_ERR_SHAPE;     // at most 0.1 s (1.6 s for the slowest waiter)
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
+    char* ws = acquire_ws(cx, COUNTER_BYTES);
+    if (!ws) return PSA_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    cudaError_t e = cudaMemsetAsync(ws, 0, 2 * COUNTER_BLOCK_BYTES, stream);
+    if (e == cudaSuccess) e = launch_wait_expiry(reinterpret_cast<DeviceCounters*>(ws), limit_us, stream);
+    if (e != cudaSuccess) { set_cuda_error(e, "psa_selftest_wait_expiry"); return PSA_ERR_CUDA; }
+    cx.clean_ws = nullptr;
+    cx.last_dc = reinterpret_cast<DeviceCounters*>(ws);
+    memset(&cx.last_useful, 0, sizeof(psa_counts));
+    return PSA_OK;
+}
+
+int psa_last_rescales(void* stream, uint64_t* rescales) {
+    if (!rescales) return PSA_ERR_NULL;
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
+    if (!cx.last_dc) return PSA_ERR_NULL;
+    DeviceCounters h;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = cudaMemcpy(&h, cx.last_dc, sizeof(h), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { set_cuda_error(e, "psa_last_rescales"); return PSA_ERR_CUDA; }
+    *rescales = h.rescales;
+    return PSA_OK;
 }
 
 size_t psa_workspace_bytes(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype,
@@ -392,42 +543,51 @@ size_t psa_workspace_bytes(int batch, int heads, int n, int d_model, int d_k, in
 }
 
 int psa_set_workspace(void* dev_ptr, size_t bytes) {
-    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
     if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255u)) return PSA_ERR_ALIGN;
-    g_ctx.user_ws = dev_ptr;
-    g_ctx.user_bytes = dev_ptr ? bytes : 0;
-    g_ctx.last_dc = nullptr;
-    g_ctx.clean_ws = nullptr;
+    cx.user_ws = dev_ptr;
+    cx.user_bytes = dev_ptr ? bytes : 0;
+    cx.last_dc = nullptr;
+    cx.clean_ws = nullptr;
     return PSA_OK;
 }
 
 int psa_profile_begin(int max_calls) {
-    std::lock_guard<std::mutex> lock(g_ctx.mu);
-    for (cudaEvent_t e : g_ctx.prof_events) cudaEventDestroy(e);
-    g_ctx.prof_events.clear();
-    g_ctx.prof_calls = 0;
-    g_ctx.prof_max = 0;
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
+    for (cudaEvent_t e : cx.prof_events) cudaEventDestroy(e);
+    cx.prof_events.clear();
+    cx.prof_calls = 0;
+    cx.prof_max = 0;
     if (max_calls <= 0 || max_calls > 100000) return PSA_ERR_SHAPE;
-    g_ctx.prof_events.resize(3 * (size_t)max_calls);
-    for (size_t i = 0; i < g_ctx.prof_events.size(); ++i) {
-        cudaError_t e = cudaEventCreate(&g_ctx.prof_events[i]);
+    cx.prof_events.resize(3 * (size_t)max_calls);
+    for (size_t i = 0; i < cx.prof_events.size(); ++i) {
+        cudaError_t e = cudaEventCreate(&cx.prof_events[i]);
         if (e != cudaSuccess) {
             set_cuda_error(e, "cudaEventCreate");
-            for (size_t k = 0; k < i; ++k) cudaEventDestroy(g_ctx.prof_events[k]);
-            g_ctx.prof_events.clear();
+            for (size_t k = 0; k < i; ++k) cudaEventDestroy(cx.prof_events[k]);
+            cx.prof_events.clear();
             return PSA_ERR_CUDA;
         }
     }
-    g_ctx.prof_max = max_calls;
+    cx.prof_max = max_calls;
     return PSA_OK;
 }
 
 int psa_profile_end(float* proj_ms_sum, float* attn_ms_sum, int* calls) {
-    std::lock_guard<std::mutex> lock(g_ctx.mu);
+    Context* cp = current_ctx();
+    if (!cp) return PSA_ERR_CUDA;
+    Context& cx = *cp;
+    std::lock_guard<std::mutex> lock(cx.mu);
     float p = 0.f, a = 0.f;
     int rc = PSA_OK;
-    for (int c = 0; c < g_ctx.prof_calls; ++c) {
-        cudaEvent_t* ev = &g_ctx.prof_events[3 * c];
+    for (int c = 0; c < cx.prof_calls; ++c) {
+        cudaEvent_t* ev = &cx.prof_events[3 * c];
         float t0 = 0.f, t1 = 0.f;
         cudaError_t e = cudaEventSynchronize(ev[2]);
         if (e == cudaSuccess) e = cudaEventElapsedTime(&t0, ev[0], ev[1]);
@@ -437,11 +597,11 @@ int psa_profile_end(float* proj_ms_sum, float* attn_ms_sum, int* calls) {
     }
     if (proj_ms_sum) *proj_ms_sum = p;
     if (attn_ms_sum) *attn_ms_sum = a;
-    if (calls) *calls = g_ctx.prof_calls;
-    for (cudaEvent_t e : g_ctx.prof_events) cudaEventDestroy(e);
-    g_ctx.prof_events.clear();
-    g_ctx.prof_calls = 0;
-    g_ctx.prof_max = 0;
+    if (calls) *calls = cx.prof_calls;
+    for (cudaEvent_t e : cx.prof_events) cudaEventDestroy(e);
+    cx.prof_events.clear();
+    cx.prof_calls = 0;
+    cx.prof_max = 0;
     return rc;
 }
 

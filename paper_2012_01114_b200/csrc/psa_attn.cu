@@ -346,13 +346,15 @@ sym_attn_kernel(const __grid_constant__ SymMaps maps, const float* __restrict__ 
                 for (int c = 0; c < NCH; ++c) {
                     uint32_t pk[16];
                     const int kc = col_base + 32 * c;            // first key column of the chunk
-                    rowsum += ragged ? exp_chunk32<0, true>(sreg[c], sl2, -m_run, kc, cb, pk)
-                                     : exp_chunk32<0, false>(sreg[c], sl2, -m_run, kc, r, pk);
+                    rowsum += ragged ? exp_chunk32<true>(sreg[c], sl2, -m_run, kc, cb, pk)
+                                     : exp_chunk32<false>(sreg[c], sl2, -m_run, kc, r, pk);
                     tmem_st16(tP + (kc >> 1), pk);
                 }
             }
             l_run = fmaf(l_run, alpha, rowsum);
             if (ok && j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8
+                const unsigned grown = __ballot_sync(0xffffffffu, alpha != 1.f);
+                if (part == 0 && lane == 0) atomicAdd(&dc->rescales, (unsigned long long)__popc(grown));
 #pragma unroll
                 for (int c = 0; c < OPT / 32; ++c) {
                     uint32_t v[32];
@@ -426,15 +428,14 @@ template <int D>
 int launch_symmetric(const void* X, void* out, float* S, int B, int H, int n, float scale, DeviceCounters* dc,
                      cudaStream_t stream) {
     using Cfg = SymCfg<D>;
-    static_assert(TPR == 2, "the symmetric kernels pair two threads per row");
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(sym_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(sym_scores_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SCORES_SMEM);
-        if (e != cudaSuccess) { set_cuda_error(e, "cudaFuncSetAttribute(symmetric attention)"); return PSA_ERR_CUDA; }
-        attr_set = true;
-    }
+    static DeviceSetup setup;
+    if (device_setup(&setup, [] {
+            cudaError_t e = cudaFuncSetAttribute(sym_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, SymCfg<D>::SMEM);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(sym_scores_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, SymCfg<D>::SCORES_SMEM);
+            return e;
+        }, "cudaFuncSetAttribute(symmetric attention)") <= 0)
+        return PSA_ERR_CUDA;
     const int T = row_tiles(n), np = sym_pairs(T);
     const int hp = sym_heads_per_pass(B, H, n);
     const uint64_t cols = (uint64_t)H * D;

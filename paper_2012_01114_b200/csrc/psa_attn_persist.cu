@@ -56,7 +56,6 @@ struct PCfg {
     static constexpr int SMEM = (2 + KSTAGES + VSTAGES) * TILE_BYTES + STAGE_BUFS * STAGE_BYTES + 1024;
     static constexpr bool SEP_P = D == 64;
     static constexpr int TMEM_S = 0, TMEM_P = 256, TMEM_O = SEP_P ? 384 : 256;
-    static constexpr int POLY_OF_4 = PSA_POLY_OF_4;
 };
 
 struct PMaps {
@@ -97,8 +96,6 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                     int group, int nitems, int split_arg, float sl2, DeviceCounters* dc, DeviceCounters* dc_next) {
     using Cfg = PCfg<D>;
     constexpr bool SEP = Cfg::SEP_P;
-    // (the experimental build with one softmax thread per row is kept working at d_k = 64 only)
-    static_assert(TPR == 2 || D == 64, "PSA_THREADS_PER_ROW=1 is not supported at d_k = 128");
     constexpr int KST = Cfg::KSTAGES, VST = Cfg::VSTAGES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -126,7 +123,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
     if (threadIdx.x == 0) {
         abort_flag = 0;
         // the counter block of the NEXT call on this workspace is cleared here, off that call's critical path
-        if (blockIdx.x == 0 && dc_next) *dc_next = DeviceCounters{0, 0, 0, 0, 0, 0};
+        if (blockIdx.x == 0 && dc_next) *dc_next = DeviceCounters{0, 0, 0, 0, 0, 0, 0};
         for (int i = 0; i < 8; ++i) stage_released[i] = 0;
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bars.item_full[t], 1);
@@ -481,7 +478,6 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                     else ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
                 }
                 ok = __all_sync(0xffffffffu, ok);
-                if (TPR == 1 && !ok) break;
                 // Element predicate: on the diagonal block of the masked scheme keys beyond the row's own index,
                 // and on a ragged last block keys beyond the sequence, carry no weight.  `cb` = last kept column.
                 const int nvalid = min(TILE, n - j * TILE);
@@ -501,14 +497,12 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                         mx = diag ? max_chunk32<true>(sreg[c], col_base + 32 * c, cb, mx)
                                   : max_chunk32<false>(sreg[c], col_base + 32 * c, r, mx);
                 }
-                if (TPR == 2) {
-                    // The two threads of a row meet here to exchange their half-row maxima (and to leave
-                    // together if either gave up a wait).
-                    xch_max[blk & 1][t][part][r] = mx;
-                    ok = named_bar_all(ok, pair_bar, 64);
-                    if (!ok) break;
-                    mx = fmaxf(mx, xch_max[blk & 1][t][part ^ 1][r]);
-                }
+                // The two threads of a row meet here to exchange their half-row maxima (and to leave
+                // together if either gave up a wait).
+                xch_max[blk & 1][t][part][r] = mx;
+                ok = named_bar_all(ok, pair_bar, 64);
+                if (!ok) break;
+                mx = fmaxf(mx, xch_max[blk & 1][t][part ^ 1][r]);
                 const float mx2 = mx * sl2;
                 float alpha = 1.f;
                 if (mx2 > m_run + RESCALE_THRESHOLD) {   // also taken on the first block (m_run = -inf)
@@ -517,11 +511,10 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                 }
                 // ---- pass 2: P = exp2(S*sl2 - m) as bf16
                 float rowsum = 0.f;
-                if (TPR == 2) {      // the scores were only reduced so far: fetch them again
+                // the scores were only reduced so far: fetch them again
 #pragma unroll
-                    for (int c = 0; c < NCH; ++c) tmem_ld32(tS + col_base + 32 * c, sreg[c]);
-                    tc_wait_ld();
-                }
+                for (int c = 0; c < NCH; ++c) tmem_ld32(tS + col_base + 32 * c, sreg[c]);
+                tc_wait_ld();
                 if (SEP) {
                     // S is in registers: the issuer may overwrite it with the next scores while the exponentials run
                     tc_fence_before();
@@ -539,14 +532,16 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                     for (int c = 0; c < NCH; ++c) {
                         uint32_t pk[16];
                         const int kc = col_base + 32 * c;            // first key column of the chunk
-                        rowsum += diag ? exp_chunk32<Cfg::POLY_OF_4, true>(sreg[c], sl2, -m_run, kc, cb, pk)
-                                       : exp_chunk32<Cfg::POLY_OF_4, false>(sreg[c], sl2, -m_run, kc, r, pk);
+                        rowsum += diag ? exp_chunk32<true>(sreg[c], sl2, -m_run, kc, cb, pk)
+                                       : exp_chunk32<false>(sreg[c], sl2, -m_run, kc, r, pk);
                         // P over S: keys [kc, kc+32) go to S columns (kc/64)*64 + (kc%64)/2, behind this thread's own reads
                         tmem_st16(SEP ? tP + (kc >> 1) : tS + (kc >> 6) * 64 + ((kc & 63) >> 1), pk);
                     }
                 }
                 l_run = fmaf(l_run, alpha, rowsum);
                 if (ok && j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8
+                    const unsigned grown = __ballot_sync(0xffffffffu, alpha != 1.f);
+                    if (part == 0 && lane == 0) atomicAdd(&dc->rescales, (unsigned long long)__popc(grown));
 #pragma unroll
                     for (int c = 0; c < OPT / 32; ++c) {
                         uint32_t v[32];
@@ -562,7 +557,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
                 mbar_arrive(&bars.p_ready[t]);
             }
             if (ok) ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
-            if (TPR == 2) xch_sum[t][part][r] = l_run;
+            xch_sum[t][part][r] = l_run;
             ok = named_bar_all(ok, pair_bar, 32 * TPR);
             if (!ok) break;
             // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row), bf16.  A unit (a warp, or
@@ -570,7 +565,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
             // TMA.  Buffers are taken in the fixed order of the units; a unit waits until the store of the unit
             // that last used its buffer has read it.
             tc_fence_after();
-            const float inv = 1.f / (TPR == 2 ? l_run + xch_sum[t][part ^ 1][r] : l_run);
+            const float inv = 1.f / (l_run + xch_sum[t][part ^ 1][r]);
             const uint32_t unit = Cfg::WARP_UNITS ? it * 16u + 8u * t + 4u * part + q : it * 8u + 4u * t + q;
             const uint32_t sbuf = unit % Cfg::STAGE_BUFS, suse = unit / Cfg::STAGE_BUFS;
             uint8_t* stage = sStage + sbuf * Cfg::STAGE_BYTES;
@@ -626,16 +621,11 @@ template <int D>
 int launch_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, float scale,
                    int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream) {
     using Cfg = PCfg<D>;
-    static bool attr_set = false;
-    static int sm_count = 0;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attn_persist_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
-        int dev = 0;
-        if (e == cudaSuccess) e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess || sm_count <= 0) { set_cuda_error(e, "attention kernel set-up"); return PSA_ERR_CUDA; }
-        attr_set = true;
-    }
+    static DeviceSetup setup;
+    const int sm_count = device_setup(&setup, [] {
+        return cudaFuncSetAttribute(attn_persist_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, PCfg<D>::SMEM);
+    }, "attention kernel set-up");
+    if (sm_count <= 0) return PSA_ERR_CUDA;
     const uint64_t cols = (uint64_t)H * D;
     PMaps maps;
     if (!make_tensor_map_bf16_3d(&maps.q, Q, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.k, K, B, n, cols, 128) ||

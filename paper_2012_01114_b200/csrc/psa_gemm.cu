@@ -268,15 +268,11 @@ gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, int
 
 int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int nW, int M, int K, int N,
                  DeviceCounters* dc, cudaStream_t stream) {
-    static int sm_count = 0;
-    if (!sm_count) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
-        int dev = 0, sms = 0;
-        if (e == cudaSuccess) e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess || sms <= 0) { set_cuda_error(e, "gemm set-up"); return PSA_ERR_CUDA; }
-        sm_count = sms;
-    }
+    static DeviceSetup setup;
+    const int sm_count = device_setup(&setup, [] {
+        return cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+    }, "gemm set-up");
+    if (sm_count <= 0) return PSA_ERR_CUDA;
     GemmMaps maps;
     if (!make_tensor_map_bf16(&maps.a, A, M, K, (uint64_t)K * 2, BM, BK)) return PSA_ERR_CUDA;
     for (int w = 0; w < 3; ++w) {

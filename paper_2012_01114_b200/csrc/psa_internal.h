@@ -16,6 +16,9 @@ struct DeviceCounters {
     unsigned long long exps;
     int status;  // PSA_OK or PSA_ERR_TIMEOUT
     unsigned int next_item;  // work-list cursor of the persistent attention kernel
+    // (row, key block) events of the bf16 online softmax in which a row's running maximum was raised after the
+    // row's first block, so that its partial output and row sum were rescaled (diagnostic, psa_last_rescales)
+    unsigned long long rescales;
 };
 
 // ---- fp32 CUDA-core path (psa_f32.cu) ----
@@ -40,6 +43,25 @@ size_t bf16_symmetric_scratch_bytes(int B, int H, int n);
 // The persistent fused kernel behind bf16_attention for PSA_FULL and PSA_MASKED (psa_attn_persist.cu).
 int bf16_attention_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, int d,
                            float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream);
+
+// Once-per-device set-up of a kernel family.  Function attributes (the dynamic shared-memory limit) belong to the
+// device that is current when they are set, and the SM count differs between devices, so both are kept per
+// device ordinal.  device_setup() returns the current device's SM count (> 0), having run `configure` (which sets
+// the family's attributes) the first time that device is seen; 0 on failure (error text set).  Thread-safe.
+constexpr int MAX_DEVICES = 64;
+struct DeviceSetup {
+    bool done[MAX_DEVICES];
+    int sm_count[MAX_DEVICES];
+};
+int device_setup(DeviceSetup* st, cudaError_t (*configure)(), const char* what);
+
+// Self-test of the bounded-wait failure path (psa_selftest.cu): a one-CTA kernel whose barrier nobody completes.
+cudaError_t launch_wait_expiry(DeviceCounters* dc, unsigned limit_us, cudaStream_t stream);
+
+// Pipe-rate measurement (psa_pipes.cu): three kernels (ex2, fma, softmax mix), each storing per SM the cycles its
+// slowest warp took for pipe_results_per_launch_per_sm() results.
+cudaError_t launch_pipe_rates(unsigned long long* cycles, float* sink, int sms, cudaStream_t stream);
+double pipe_results_per_launch_per_sm();
 
 void set_cuda_error(cudaError_t e, const char* where);
 void set_error_text(const char* text);

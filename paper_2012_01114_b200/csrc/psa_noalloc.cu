@@ -12,6 +12,8 @@
 // the process exits, the problem size is capped, and all calls share the one array.
 #include <stdio.h>
 
+#include <mutex>
+
 #include "psa_internal.h"
 
 namespace psa {
@@ -27,8 +29,8 @@ static_assert(sizeof(DeviceCounters) <= NOALLOC_COUNTER_BYTES, "counter block to
 // name is only a handle for the runtime's symbol table; the device address is looked up below.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
 
-constexpr int MAX_DEVICES = 64;
 unsigned char* g_scratch_addr[MAX_DEVICES];  // device address of the array, per device ordinal (0 = not looked up)
+std::mutex g_scratch_mu;                     // guards the table above
 
 }  // namespace
 }  // namespace psa
@@ -37,6 +39,7 @@ using namespace psa;
 
 extern "C" int psa_attention_sym_f32_noalloc(const void* X, int batch, int heads, int n, int d_k, void* out,
                                              void* stream_v) {
+    set_error_text("");
     if (!X || !out) return PSA_ERR_NULL;
     if (batch <= 0 || heads <= 0 || n <= 0 || d_k <= 0) return PSA_ERR_SHAPE;
     if (n > 1024 || d_k > 128) return PSA_ERR_UNSUPPORTED;
@@ -54,13 +57,17 @@ extern "C" int psa_attention_sym_f32_noalloc(const void* X, int batch, int heads
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) { set_cuda_error(e, "cudaGetDevice"); return PSA_ERR_CUDA; }
     if (dev < 0 || dev >= MAX_DEVICES) return PSA_ERR_UNSUPPORTED;
-    if (!g_scratch_addr[dev]) {  // first call on this device: resolve the array's device address
-        unsigned char* p = nullptr;
-        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_scratch);
-        if (e != cudaSuccess || !p) { set_cuda_error(e, "cudaGetSymbolAddress(scratch)"); return PSA_ERR_CUDA; }
-        g_scratch_addr[dev] = p;
+    unsigned char* base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_scratch_mu);
+        if (!g_scratch_addr[dev]) {  // first call on this device: resolve the array's device address
+            unsigned char* p = nullptr;
+            e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_scratch);
+            if (e != cudaSuccess || !p) { set_cuda_error(e, "cudaGetSymbolAddress(scratch)"); return PSA_ERR_CUDA; }
+            g_scratch_addr[dev] = p;
+        }
+        base = g_scratch_addr[dev];
     }
-    unsigned char* base = g_scratch_addr[dev];
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     DeviceCounters* dc = reinterpret_cast<DeviceCounters*>(base);
     // The array keeps what the previous call left.  The counters must start at zero; the score region

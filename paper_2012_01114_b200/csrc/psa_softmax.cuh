@@ -6,15 +6,8 @@
 
 namespace psa {
 
-#ifndef PSA_POLY_OF_4
-#define PSA_POLY_OF_4 0
-#endif
-#ifndef PSA_THREADS_PER_ROW
-#define PSA_THREADS_PER_ROW 2
-#endif
-
 constexpr int CTRL_WARPS = 2;                       // producer, MMA issuer
-constexpr int TPR = PSA_THREADS_PER_ROW;            // softmax threads per query row: 2 (1 is an experiment, d_k = 64 only, slower)
+constexpr int TPR = 2;                              // softmax threads per query row (each owns 64 of a block's 128 columns)
 constexpr int SOFTMAX_WARPS_PER_TILE = 4 * TPR;
 constexpr int ATTN_THREADS = 32 * (CTRL_WARPS + 2 * SOFTMAX_WARPS_PER_TILE);   // 576
 constexpr float LOG2E = 1.4426950408889634f;
@@ -25,18 +18,6 @@ __device__ __forceinline__ float ex2_mufu(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// 2^x for x <= ~8 on the FMA pipe: n = round(x) by adding 1.5*2^23, f = x - n in [-0.5, 0.5],
-// 2^f by a cubic fitted to relative error 8e-5, then n is added into the exponent field.
-__device__ __forceinline__ float ex2_poly(float x) {
-    const float magic = 12582912.0f;
-    x = fmaxf(x, -126.0f);
-    const float t = __fadd_rn(x, magic);
-    const float f = __fsub_rn(x, __fsub_rn(t, magic));
-    float p = fmaf(f, 0.05508868396282196f, 0.24260404706001282f);
-    p = fmaf(p, f, 0.6932762265205383f);
-    p = fmaf(p, f, 0.9999289512634277f);
-    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
-}
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -46,7 +27,7 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // exp2 of 32 scores of one row (raw, unscaled) against the running maximum: P = exp2(s*sl2 - m), packed
 // to bf16 pairs in `pk`; returns the sum of the 32 weights (before rounding).  `col0` is the column of
 // s[0] inside the 128-wide block; with DIAG, columns beyond `r` carry no weight.
-template <int POLY_OF_4, bool DIAG>
+template <bool DIAG>
 __device__ __forceinline__ float exp_chunk32(const uint32_t (&s)[32], float sl2, float neg_m, int col0, int r,
                                              uint32_t (&pk)[16]) {
     float sum0 = 0.f, sum1 = 0.f;
@@ -54,8 +35,8 @@ __device__ __forceinline__ float exp_chunk32(const uint32_t (&s)[32], float sl2,
     for (int i = 0; i < 32; i += 2) {
         const float x0 = fmaf(__uint_as_float(s[i]), sl2, neg_m);
         const float x1 = fmaf(__uint_as_float(s[i + 1]), sl2, neg_m);
-        float p0 = ((i & 3) < POLY_OF_4) ? ex2_poly(x0) : ex2_mufu(x0);
-        float p1 = (((i + 1) & 3) < POLY_OF_4) ? ex2_poly(x1) : ex2_mufu(x1);
+        float p0 = ex2_mufu(x0);
+        float p1 = ex2_mufu(x1);
         if (DIAG) {
             if (col0 + i > r) p0 = 0.f;
             if (col0 + i + 1 > r) p1 = 0.f;

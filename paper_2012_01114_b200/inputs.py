@@ -72,11 +72,18 @@ def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
 
 
-def tensor(seed: int, tensor_id: int, shape, scale: float, dtype: str):
+def tensor(seed: int, tensor_id: int, shape, scale: float, dtype: str, row_scale=None):
     """Returns (values, bits): float64 values exactly representable in `dtype`, and for bf16 the
-    uint16 bit patterns to upload (for f32, a float32 array to upload)."""
+    uint16 bit patterns to upload (for f32, a float32 array to upload).
+
+    `row_scale`, if given, is one extra factor per index of axis 1 (the sequence position of a
+    [batch, n, ...] tensor), applied before the rounding to `dtype`: inputs whose magnitude varies
+    along the sequence, for instance keys that grow from one 128-key block to the next."""
     count = int(np.prod(shape))
     x = normal(seed, tensor_id, count) * scale
+    if row_scale is not None:
+        rs = np.asarray(row_scale, dtype=np.float64)
+        x = (x.reshape(shape[0], shape[1], -1) * rs[None, :, None]).reshape(-1)
     if dtype == "bf16":
         bits = to_bf16_bits(x).reshape(shape)
         return bf16_bits_to_f64(bits), bits

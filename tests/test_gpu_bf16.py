@@ -164,3 +164,17 @@ def test_host_entry_matches_device_entry():
     binding.psa_attention_host(*host, H, binding.MASKED, out_h)
     out_d = binding.psa_attention(*[t.cuda() for t in host], H, binding.MASKED)
     assert torch.equal(out_h.view(torch.int16), out_d.cpu().view(torch.int16))
+
+
+def test_core_host_entry_matches_device_entry():
+    B, H, n, d = 2, 2, 300, 128
+    bits = [inputs.tensor(19, t, (B, n, H, d), 1.0, "bf16")[1] for t in (4, 5, 6)]
+    host = [torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) for a in bits]
+    for scheme in (binding.FULL, binding.MASKED, binding.SYMMETRIC):
+        sym = scheme == binding.SYMMETRIC
+        out_h = torch.empty((B, n, H * d), dtype=torch.bfloat16)
+        binding.psa_attention_core_host(host[0], None if sym else host[1], None if sym else host[2], scheme, out_h)
+        _check_census(B, H, n, 0, d, scheme)
+        out_d = binding.psa_attention_core(host[0].cuda(), None if sym else host[1].cuda(),
+                                           None if sym else host[2].cuda(), scheme)
+        assert torch.equal(out_h.view(torch.int16), out_d.cpu().view(torch.int16))

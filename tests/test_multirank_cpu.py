@@ -29,9 +29,16 @@ def _rank_main(rank, world, port, out_path):
     t = torch.tensor([my_seconds], dtype=torch.float64)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     value = bench.aggregate([my_flops] * world, float(t.item()))
+    # the decision to take another round of steps is taken on the least advanced rank's time, the same everywhere:
+    # rank 0 has 1200 ms, rank 1 only 900 ms of a 1 s region -> both go on; at 1200 / 1100 ms both stop
+    go_on = bench.more_rounds(1200.0 - 300.0 * rank, 3, 1.0, 100, dist)
+    stop = bench.more_rounds(1200.0 - 100.0 * rank, 4, 1.0, 100, dist)
+    capped = bench.more_rounds(10.0, 100, 1.0, 100, dist)
+    decisions = [None] * world
+    dist.all_gather_object(decisions, (go_on, stop, capped))
     if rank == 0:
         with open(out_path, "w") as f:
-            json.dump({"value": value, "max_seconds": float(t.item())}, f)
+            json.dump({"value": value, "max_seconds": float(t.item()), "decisions": decisions}, f)
     dist.destroy_process_group()
 
 
@@ -42,6 +49,7 @@ def test_two_rank_timing_protocol(tmp_path):
     got = json.load(open(out))
     assert got["max_seconds"] == pytest.approx(0.75)
     assert got["value"] == pytest.approx(2 * 3.0 / 0.75)      # TFLOP/s: both ranks' work over the slowest time
+    assert got["decisions"] == [[True, False, False], [True, False, False]]
 
 
 def test_useful_flops_formulas_match_the_papers_counts():

@@ -4,8 +4,9 @@ It serves callers that are not allowed to allocate device memory while running (
 plug-ins that do not own the allocator, latency-critical loops), so its scratch is an array built into
 the library.  This test calls it through the C interface twice in a row -- the second call finds the
 array dirty from the first -- and checks each result against the regular entry point
-(psa_attention_core, symmetric scheme, fp32) within the fp32 tolerance of the other GPU tests, and the
-size limit's error.  The file name sorts last so that a run stopping at the first failure has already
+(psa_attention_core, symmetric scheme, fp32) and against the fp64 oracle within the fp32 tolerance of the
+other GPU tests, that the device's free memory is the same before and after a call, and the size limit's
+error.  The file name sorts last so that a run stopping at the first failure has already
 run everything else; the test also passes on its own in a fresh process.
 """
 import ctypes
@@ -14,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2012_01114_b200 import binding
 
 pytestmark = pytest.mark.gpu
@@ -41,9 +43,28 @@ def test_noalloc_matches_regular_entry_on_two_calls_in_a_row():
         ref = binding.psa_attention_core(X, None, None, binding.SYMMETRIC)
         err = (out - ref).abs().max().item()
         assert err <= TOL_F32, err
+        x64 = X.cpu().numpy().astype(np.float64)
+        want, _ = oracle.attention_core(x64, x64, x64, oracle.SYMMETRIC)
+        assert np.abs(out.cpu().numpy().astype(np.float64) - want).max() <= TOL_F32
     # same input again through the Python wrapper: the dirty scratch must not leak into the result
     again = binding.psa_attention_sym_f32_noalloc(cases[0][0])
     assert (again - outs[0]).abs().max().item() <= TOL_F32
+
+
+def test_noalloc_call_leaves_free_device_memory_unchanged():
+    # the property the entry point exists for: with the output tensor made beforehand, a call changes nothing
+    # about the device's memory (the first call on a device, which looks up the array's address, came earlier)
+    X = _x(5, (1, 128, 2, 32))
+    out = torch.empty((1, 128, 64), dtype=torch.float32, device="cuda")
+    stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    args = (ctypes.c_void_p(X.data_ptr()), 1, 2, 128, 32, ctypes.c_void_p(out.data_ptr()), stream)
+    assert binding.lib().psa_attention_sym_f32_noalloc(*args) == binding.OK
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for _ in range(3):
+        assert binding.lib().psa_attention_sym_f32_noalloc(*args) == binding.OK
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
 
 
 def test_noalloc_rejects_problems_beyond_its_scratch():
