@@ -419,14 +419,15 @@ int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme
     // same block lists taken one at a time: the census does not depend on the grouping.)
     const int T = row_tiles(n);
     const uint64_t block_macs = (uint64_t)TILE * TILE * d_k;
-    uint64_t qk_blocks = 0, pv_blocks = 0;
+    uint64_t qk_blocks = 0, pv_blocks = 0, exps = 0;
     const int P = ctas_per_head(n);
     for (int cta = 0; cta < P; ++cta) {  // every head has the same list
         const CtaWork w = cta_work(cta, n, scheme == PSA_MASKED, 1, 1);
         for (int t = 0; t < w.ntiles; ++t) {
-            const int kv = kv_tiles(w.tile0 + t, T, scheme);
+            const int I = w.tile0 + t, kv = kv_tiles(I, T, scheme);
             pv_blocks += kv;
             if (scheme != PSA_SYMMETRIC) qk_blocks += kv;
+            exps += (uint64_t)kv * TILE * TILE;      // every weight of an issued block is exponentiated
         }
     }
     if (scheme == PSA_SYMMETRIC) {
@@ -438,7 +439,7 @@ int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme
     }
     c->qk_macs = bh * qk_blocks * block_macs;
     c->pv_macs = bh * pv_blocks * block_macs;
-    c->exps = bh * pv_blocks * (uint64_t)TILE * TILE;
+    c->exps = bh * exps;
     return PSA_OK;
 }
 

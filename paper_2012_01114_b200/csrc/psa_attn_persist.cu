@@ -92,8 +92,8 @@ template <int D> __host__ __device__ constexpr int item_readers() { return (D ==
 
 template <int D>
 __global__ void __launch_bounds__(persist_threads<D>(), 1)
-attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme, int nbh,
-                    int group, int nitems, int split_arg, float sl2, DeviceCounters* dc, DeviceCounters* dc_next) {
+attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ SchedParams sp, int H, int scheme,
+                    int nitems, float sl2, DeviceCounters* dc, DeviceCounters* dc_next) {
     using Cfg = PCfg<D>;
     constexpr bool SEP = Cfg::SEP_P;
     constexpr int KST = Cfg::KSTAGES, VST = Cfg::VSTAGES;
@@ -112,13 +112,11 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, int n, int H, int scheme
     __shared__ float xch_sum[2][2][128];      // [tile][column half][row]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int T = row_tiles(n);
-    const int masked = scheme == PSA_MASKED;
-    // single-tile items at the end of the list exist at d = 64 only (a lone row tile gains nothing at d = 128)
-    auto item_work = [&](int idx) -> CtaWork {
-        if constexpr (D == 64) return cta_work_split(idx, n, masked, nbh, group, split_arg);
-        else return cta_work(idx, n, masked, nbh, group);
-    };
+    const int n = sp.n, T = sp.T;
+    const int masked = sp.masked;
+    // An item index is decoded without divisions (psa_sched.h); single-tile items at the end of the list exist at
+    // d = 64 only (a lone row tile gains nothing at d = 128: the host puts split_from beyond the list there).
+    auto item_work = [&](int idx) -> CtaWork { return item_work_fast(sp, idx); };
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -636,9 +634,10 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
     const long long nitems = pairs + (pairs - split);          // pairs, then the rest as single row tiles
     if (nitems > 0x7fffffffLL - sm_count) return PSA_ERR_SHAPE;
     const int grid = (int)(nitems < sm_count ? nitems : sm_count);
-    attn_persist_kernel<D><<<grid, persist_threads<D>(), Cfg::SMEM, stream>>>(
-        maps, n, H, scheme, B * H, lpt_group(scheme, B * H, n, D), (int)nitems,
-        split == pairs ? 0x7fffffff : (int)split, scale * LOG2E, dc, dc_next);
+    const SchedParams sp = sched_params(n, scheme == PSA_MASKED, B * H, lpt_group(scheme, B * H, n, D),
+                                        split == pairs ? 0x7fffffff : (int)split);
+    attn_persist_kernel<D><<<grid, persist_threads<D>(), Cfg::SMEM, stream>>>(maps, sp, H, scheme, (int)nitems,
+                                                                            scale * LOG2E, dc, dc_next);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "attn_persist_kernel launch"); return PSA_ERR_CUDA; }
     return PSA_OK;

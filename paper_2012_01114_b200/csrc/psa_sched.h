@@ -21,6 +21,37 @@ namespace psa {
 constexpr int TILE = 128;          // rows and columns of one block of the weight matrix
 constexpr int TILES_PER_CTA = 2;   // a CTA owns two consecutive row tiles of one (batch, head)
 
+// Division of a 32-bit unsigned number by a divisor fixed for a whole launch, as a multiply-high and two shifts
+// (the kernels decode a work-item index several thousand times per CTA; the hardware has no integer divide, and
+// the compiler's general sequence costs a single thread several hundred cycles per item).  For d >= 2:
+//     l = ceil(log2 d),  m = floor(2^32 (2^l - d) / d) + 1,  n / d = (t + ((n - t) >> 1)) >> (l - 1),  t = hi32(m n)
+// exact for every 32-bit n (the round-up method with a 33-bit multiplier, its top bit folded into the second shift).
+struct FastDiv {
+    uint32_t d, m, s;      // divisor, multiplier, l - 1   (d = 1: m = 0, s = 0 and the quotient is n itself)
+};
+PSA_HD FastDiv fastdiv_make(uint32_t d) {
+    FastDiv f;
+    f.d = d; f.m = 0; f.s = 0;
+    if (d <= 1) return f;
+    uint32_t l = 0;
+    while ((1ull << l) < d) ++l;
+    f.m = (uint32_t)(((1ull << 32) * ((1ull << l) - d)) / d + 1);
+    f.s = l - 1;
+    return f;
+}
+PSA_HD uint32_t fastdiv_hi32(uint32_t a, uint32_t b) {
+#if defined(__CUDA_ARCH__)
+    return __umulhi(a, b);
+#else
+    return (uint32_t)(((uint64_t)a * b) >> 32);
+#endif
+}
+PSA_HD uint32_t fastdiv(uint32_t n, const FastDiv& f) {
+    if (f.d <= 1) return n;
+    const uint32_t t = fastdiv_hi32(f.m, n);
+    return (t + ((n - t) >> 1)) >> f.s;
+}
+
 struct CtaWork {
     int bh;        // batch * heads + head
     int tile0;     // first row tile owned
@@ -61,6 +92,48 @@ PSA_HD CtaWork cta_work_split(int item, int n, int scheme_masked, int nbh, int g
     w.ntiles = 1;
     return w;
 }
+// The same decoding with every division replaced by FastDiv: the launch's constants are prepared once on the host.
+struct SchedParams {
+    int n, masked, nbh, group, P, T, full_groups, tail, split_from;
+    FastDiv by_group_items;   // / (group * P)
+    FastDiv by_group;         // / group
+    FastDiv by_tail;          // / tail   (heads in the last, partial group; 0 if none)
+};
+PSA_HD SchedParams sched_params(int n, int scheme_masked, int nbh, int group, int split_from) {
+    SchedParams sp;
+    sp.n = n; sp.masked = scheme_masked; sp.nbh = nbh; sp.group = group; sp.split_from = split_from;
+    sp.P = ctas_per_head(n); sp.T = row_tiles(n);
+    sp.full_groups = nbh / group;
+    sp.tail = nbh - sp.full_groups * group;
+    sp.by_group_items = fastdiv_make((uint32_t)group * (uint32_t)sp.P);
+    sp.by_group = fastdiv_make((uint32_t)group);
+    sp.by_tail = fastdiv_make((uint32_t)(sp.tail > 0 ? sp.tail : 1));
+    return sp;
+}
+PSA_HD CtaWork cta_work_fast(const SchedParams& sp, int cta) {
+    int g = (int)fastdiv((uint32_t)cta, sp.by_group_items);
+    if (g > sp.full_groups) g = sp.full_groups;
+    const int off = cta - g * sp.group * sp.P;
+    const bool full = g < sp.full_groups;
+    const int size = full ? sp.group : sp.tail;
+    const int r = (int)fastdiv((uint32_t)off, full ? sp.by_group : sp.by_tail);
+    CtaWork w;
+    w.bh = g * sp.group + (off - r * size);
+    const int p = sp.masked ? (sp.P - 1 - r) : r;
+    w.tile0 = p * TILES_PER_CTA;
+    const int left = sp.T - w.tile0;
+    w.ntiles = left < TILES_PER_CTA ? left : TILES_PER_CTA;
+    return w;
+}
+// ... and with the tail of single row tiles (cta_work_split)
+PSA_HD CtaWork item_work_fast(const SchedParams& sp, int item) {
+    if (item < sp.split_from) return cta_work_fast(sp, item);
+    CtaWork w = cta_work_fast(sp, sp.split_from + ((item - sp.split_from) >> 1));
+    w.tile0 += (item - sp.split_from) & 1;
+    w.ntiles = 1;
+    return w;
+}
+
 // Work items of a launch over `pairs` pairs of row tiles on `sms` persistent CTAs: the first split_point() items are
 // pairs, the rest single row tiles.  Where all CTAs do the same work (FULL) and the last round of pairs would occupy
 // at most half of the CTAs, those pairs are handed out as single tiles instead, so that twice as many CTAs share

@@ -50,19 +50,22 @@ __device__ __forceinline__ float exp_chunk32(const uint32_t (&s)[32], float sl2,
 
 template <bool DIAG>
 __device__ __forceinline__ float max_chunk32(const uint32_t (&s)[32], int col0, int r, float mx) {
-    if (!DIAG) {
-        float a = mx, b = -INFINITY;
+    // four independent accumulators: the chain of dependent maxima is 4 long, not 16 (the three-input maximum has a
+    // latency of about a dozen cycles); with DIAG, columns beyond `r` are replaced by -inf first
+    float a[4] = {mx, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-            a = max3(a, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
-            b = max3(b, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+    for (int i = 0; i < 32; i += 8) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float x0 = __uint_as_float(s[i + 2 * k]), x1 = __uint_as_float(s[i + 2 * k + 1]);
+            if (DIAG) {
+                if (col0 + i + 2 * k > r) x0 = -INFINITY;
+                if (col0 + i + 2 * k + 1 > r) x1 = -INFINITY;
+            }
+            a[k] = max3(a[k], x0, x1);
         }
-        return fmaxf(a, b);
     }
-#pragma unroll
-    for (int i = 0; i < 32; ++i)
-        if (col0 + i <= r) mx = fmaxf(mx, __uint_as_float(s[i]));
-    return mx;
+    return fmaxf(max3(a[0], a[1], a[2]), a[3]);
 }
 
 }  // namespace psa

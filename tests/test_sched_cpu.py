@@ -22,9 +22,12 @@ int main(int argc, char** argv) {
     const int group = lpt_group(scheme, nbh, n, d);
     std::vector<int> seen((size_t)nbh * T, 0);
     long long singles = 0;
+    const SchedParams sp = sched_params(n, scheme == PSA_MASKED, nbh, group, split == pairs ? 0x7fffffff : (int)split);
     for (long long i = 0; i < nitems; ++i) {
         const CtaWork w = split == pairs ? cta_work((int)i, n, scheme == PSA_MASKED, nbh, group)
                                          : cta_work_split((int)i, n, scheme == PSA_MASKED, nbh, group, (int)split);
+        const CtaWork f = item_work_fast(sp, (int)i);      // the division-free decoding the kernel uses
+        if (f.bh != w.bh || f.tile0 != w.tile0 || f.ntiles != w.ntiles) return 5;
         if (w.bh < 0 || w.bh >= nbh || w.ntiles < 1 || w.ntiles > 2 || w.tile0 < 0 || w.tile0 + w.ntiles > T) return 2;
         if (i >= split && w.ntiles != 1) return 3;
         if (i >= split) ++singles;
