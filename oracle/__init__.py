@@ -181,17 +181,22 @@ def attention_layer(X, Wq, Wk, Wv, heads, scheme, scale=None, selection=SEL_MINI
 
 
 def attention_block(X, Wq, Wk, Wv, Wo, heads, scheme, scale=None, selection=SEL_MINIMAL, round_qkv_bf16=False,
-                    round_y_bf16=False):
+                    round_y_bf16=False, residual=None):
     """The layer followed by the output projection: z = concat_h(y^(h)) * Wo, Wo [heads*d, d_model].
 
     The paper stops at y (Sec. 3.2) and names the complete model as future work (Sec. 7); this is the
     standard multi-head closing step, written as one more projection of the kind Sec. 3.1 calls a typical
     matrix-vector product.  round_y_bf16 rounds y before the product (a bf16 pipeline stores y in bf16).
+    `residual` [B, n, d_model], if given, is added to the product elementwise (the skip connection a transformer
+    block wraps around its attention sub-layer; usually X itself): z = residual + concat_h(y^(h)) * Wo.
     Returns (z [B, n, d_model], y [B, n, heads*d], Counts of the three phases)."""
     y, cnt = attention_layer(X, Wq, Wk, Wv, heads, scheme, scale, selection, round_qkv_bf16)
     if round_y_bf16:
         y = round_bf16(y)
-    return project(y, Wo), y, cnt
+    z = project(y, Wo)
+    if residual is not None:
+        z = z + _f64(residual).reshape(z.shape)
+    return z, y, cnt
 
 
 def tile_counts(n, d, scheme, bm, bn, selection=SEL_MINIMAL):

@@ -260,6 +260,30 @@ def test_block_special_output_matrices():
     assert np.abs(zm[0, 0] - (X[0, 0] @ Wv) @ A).max() <= 1e-13
 
 
+def test_block_residual_is_added_elementwise():
+    # z = residual + y Wo: with a zero output matrix the block returns the residual itself; with the residual moved to
+    # the other side it is the block without one; a library sum-of-heads product plus X pins the usual case R = X
+    rng = np.random.default_rng(8)
+    B, n, D, H, d = 2, 6, 5, 2, 3
+    X = rng.standard_normal((B, n, D)) * 0.5
+    Wq, Wk, Wv = (rng.standard_normal((D, H * d)) * 0.5 for _ in range(3))
+    Wo = rng.standard_normal((H * d, D)) * 0.5
+    R = rng.standard_normal((B, n, D))
+    z0, _, _ = oracle.attention_block(X, Wq, Wk, Wv, np.zeros((H * d, D)), H, oracle.MASKED, residual=R)
+    assert np.array_equal(z0, R)
+    z_plain, _, _ = oracle.attention_block(X, Wq, Wk, Wv, Wo, H, oracle.FULL)
+    z_res, _, _ = oracle.attention_block(X, Wq, Wk, Wv, Wo, H, oracle.FULL, residual=R)
+    assert np.abs((z_res - R) - z_plain).max() <= 1e-15
+    z_x, _, _ = oracle.attention_block(X, Wq, Wk, Wv, Wo, H, oracle.FULL, residual=X)
+    for b in range(B):
+        want = X[b].copy()
+        for h in range(H):
+            sl = slice(h * d, (h + 1) * d)
+            s_ = (X[b] @ Wq[:, sl]) @ (X[b] @ Wk[:, sl]).T / math.sqrt(d)
+            want += (scipy.special.softmax(s_, axis=1) @ (X[b] @ Wv[:, sl])) @ Wo[sl, :]
+        assert np.abs(z_x[b] - want).max() <= 1e-12
+
+
 def test_bf16_rounding_agrees_with_generator_and_torch():
     import torch
     rng = np.random.default_rng(5)
