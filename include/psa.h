@@ -131,6 +131,18 @@ int psa_attention_core_host(const void* Q_host, const void* K_host, const void* 
  */
 int psa_attention_block(const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Wo, int batch,
                         int heads, int n, int d_model, int d_k, int scheme, int dtype, void* out, void* stream);
+/*
+ * The attention block with a residual input (the skip connection a transformer block wraps around its attention
+ * sub-layer; the paper leaves the complete model to future work, Sec. 7):
+ *     z[b, i, :] = R[b, i, :] + sum_h y^(h)[b, i, :] * Wo[h*d_k : (h+1)*d_k, :].
+ *   R   device, [batch, n, d_model] row-major, same type as the other tensors, caller-owned, read only; usually X
+ *       itself; NULL gives psa_attention_block.  R must not be `out` (PSA_ERR_SCHEME_ARGS).
+ * The sum is formed in fp32 in the epilogue of the output projection, before the rounding to the storage type.
+ * Everything else as for psa_attention_block.
+ */
+int psa_attention_block_residual(const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Wo,
+                                 const void* R, int batch, int heads, int n, int d_model, int d_k, int scheme,
+                                 int dtype, void* out, void* stream);
 size_t psa_block_workspace_bytes(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype);
 
 /*

@@ -23,7 +23,7 @@ LIB_PATH = os.path.join(_HERE, "libpsa.so")
 EXPORTS = ("psa_attention", "psa_attention_f32", "psa_attention_core", "psa_attention_host", "psa_skip_count",
            "psa_last_issued", "psa_workspace_bytes", "psa_set_workspace", "psa_status_string",
            "psa_last_cuda_error", "psa_profile_begin", "psa_profile_end", "psa_attention_sym_f32_noalloc",
-           "psa_attention_block", "psa_block_workspace_bytes", "psa_last_rescales", "psa_selftest_wait_expiry", "psa_measure_pipe_rates", "psa_attention_core_host")
+           "psa_attention_block", "psa_block_workspace_bytes", "psa_last_rescales", "psa_selftest_wait_expiry", "psa_measure_pipe_rates", "psa_attention_core_host", "psa_attention_block_residual")
 
 
 class PsaError(RuntimeError):
@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.psa_profile_end.restype = ci
         L.psa_attention_block.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp]
         L.psa_attention_block.restype = ci
+        L.psa_attention_block_residual.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp]
+        L.psa_attention_block_residual.restype = ci
         L.psa_block_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ci, ci]
         L.psa_block_workspace_bytes.restype = ctypes.c_size_t
         L.psa_attention_core_host.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, vp]
@@ -194,7 +196,7 @@ def psa_attention_core_host(Q, K, V, scheme, out, stream=None):
     rc = lib().psa_attention_core_host(_ptr(Q), _ptr(K), _ptr(V), B, H, n, d, int(scheme), code, _ptr(out),
                                        _stream(stream))
     if rc != OK:
-        raise PsaError(rc, "psa_attention_core_host")
+        raise PsaError(rc, "psa_attention_core_host", "psa_attention_block_residual")
     return out
 
 
@@ -221,7 +223,7 @@ def psa_measure_pipe_rates(stream=None) -> dict:
     r = PipeRates()
     rc = lib().psa_measure_pipe_rates(ctypes.byref(r), _stream(stream))
     if rc != OK:
-        raise PsaError(rc, "psa_measure_pipe_rates", "psa_attention_core_host")
+        raise PsaError(rc, "psa_measure_pipe_rates", "psa_attention_core_host", "psa_attention_block_residual")
     return {k: getattr(r, k) for k, _ in r._fields_}
 
 
@@ -237,16 +239,16 @@ def psa_last_rescales(stream=None) -> int:
     v = ctypes.c_uint64()
     rc = lib().psa_last_rescales(_stream(stream), ctypes.byref(v))
     if rc != OK:
-        raise PsaError(rc, "psa_last_rescales", "psa_selftest_wait_expiry", "psa_measure_pipe_rates", "psa_attention_core_host")
+        raise PsaError(rc, "psa_last_rescales", "psa_selftest_wait_expiry", "psa_measure_pipe_rates", "psa_attention_core_host", "psa_attention_block_residual")
     return int(v.value)
 
 
-def psa_attention_block(X, Wq, Wk, Wv, Wo, heads, scheme, out=None, stream=None):
-    """Projections + attention + output projection.  X [B,n,D], W* [D,heads*d_k], Wo [heads*d_k,D] -> out [B,n,D]
-    (all bf16 or all fp32, CUDA)."""
+def psa_attention_block(X, Wq, Wk, Wv, Wo, heads, scheme, out=None, stream=None, residual=None):
+    """Projections + attention + output projection (+ residual).  X [B,n,D], W* [D,heads*d_k], Wo [heads*d_k,D],
+    residual [B,n,D] or None -> out [B,n,D] (all bf16 or all fp32, CUDA)."""
     dtype = X.dtype
     code = {torch.bfloat16: BF16, torch.float32: F32}[dtype]
-    for t, nm in ((X, "X"), (Wq, "Wq"), (Wk, "Wk"), (Wv, "Wv"), (Wo, "Wo"), (out, "out")):
+    for t, nm in ((X, "X"), (Wq, "Wq"), (Wk, "Wk"), (Wv, "Wv"), (Wo, "Wo"), (out, "out"), (residual, "residual")):
         _check_dev(t, dtype, nm)
     batch, n, d_model = X.shape
     hd = Wq.shape[1]
@@ -254,8 +256,15 @@ def psa_attention_block(X, Wq, Wk, Wv, Wo, heads, scheme, out=None, stream=None)
         raise ValueError("Wq must be [d_model, heads*d_k] and Wo [heads*d_k, d_model]")
     if out is None:
         out = torch.empty((batch, n, d_model), dtype=dtype, device=X.device)
-    rc = lib().psa_attention_block(_ptr(X), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(Wo), batch, heads, n, d_model,
-                                   hd // heads, int(scheme), code, _ptr(out), _stream(stream))
+    if residual is not None and tuple(residual.shape) != (batch, n, d_model):
+        raise ValueError("residual must be [batch, n, d_model]")
+    if residual is None:
+        rc = lib().psa_attention_block(_ptr(X), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(Wo), batch, heads, n, d_model,
+                                       hd // heads, int(scheme), code, _ptr(out), _stream(stream))
+    else:
+        rc = lib().psa_attention_block_residual(_ptr(X), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(Wo), _ptr(residual),
+                                                batch, heads, n, d_model, hd // heads, int(scheme), code, _ptr(out),
+                                                _stream(stream))
     if rc != OK:
         raise PsaError(rc, "psa_attention_block")
     return out

@@ -163,10 +163,10 @@ int run_layer(Context& cx, const void* X, const void* Wq, const void* Wk, const 
         const void* Ws[3] = {Wq, nW == 3 ? Wk : Wq, nW == 3 ? Wv : Wq};
         if (dtype == PSA_F32) {
             e = f32_project(static_cast<const float*>(X), reinterpret_cast<const float* const*>(Ws),
-                            reinterpret_cast<float* const*>(outs), nW, batch * n, d_model, heads * d_k, dc, stream);
+                            reinterpret_cast<float* const*>(outs), nW, batch * n, d_model, heads * d_k, nullptr, dc, stream);
             if (e != cudaSuccess) { set_cuda_error(e, "f32_project"); return PSA_ERR_CUDA; }
         } else {
-            int rc = bf16_project(X, Ws, outs, nW, batch * n, d_model, heads * d_k, dc, stream);
+            int rc = bf16_project(X, Ws, outs, nW, batch * n, d_model, heads * d_k, nullptr, dc, stream);
             if (rc != PSA_OK) return rc;
         }
         Q = ws + L.q; K = ws + L.k; V = ws + L.v;
@@ -355,6 +355,13 @@ int psa_attention_core_host(const void* Q_host, const void* K_host, const void* 
 
 int psa_attention_block(const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Wo, int batch,
                         int heads, int n, int d_model, int d_k, int scheme, int dtype, void* out, void* stream_v) {
+    return psa_attention_block_residual(X, Wq, Wk, Wv, Wo, nullptr, batch, heads, n, d_model, d_k, scheme, dtype, out,
+                                        stream_v);
+}
+
+int psa_attention_block_residual(const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Wo,
+                                 const void* R, int batch, int heads, int n, int d_model, int d_k, int scheme,
+                                 int dtype, void* out, void* stream_v) {
     g_err_text[0] = 0;
     int rc = check_shape(batch, heads, n, d_model, d_k, scheme, dtype, true);
     if (rc != PSA_OK) return rc;
@@ -364,8 +371,10 @@ int psa_attention_block(const void* X, const void* Wq, const void* Wk, const voi
     } else if (!Wk || !Wv) {
         return PSA_ERR_NULL;
     }
-    if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(Wo) || !aligned16(out))
+    if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(Wo) || !aligned16(out) ||
+        !aligned16(R))
         return PSA_ERR_ALIGN;
+    if (R == out) return PSA_ERR_SCHEME_ARGS;      // the residual is read while the output is written
     if (dtype == PSA_BF16 && (heads * d_k) % 64 != 0) return PSA_ERR_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     Context* cp = current_ctx();
@@ -387,11 +396,11 @@ int psa_attention_block(const void* X, const void* Wq, const void* Wk, const voi
     if (dtype == PSA_F32) {
         cudaError_t e = f32_project(static_cast<const float*>(y), reinterpret_cast<const float* const*>(Ws),
                                     reinterpret_cast<float* const*>(outs), 1, batch * n, heads * d_k, d_model,
-                                    cx.last_dc, stream);
+                                    static_cast<const float*>(R), cx.last_dc, stream);
         if (e != cudaSuccess) { set_cuda_error(e, "f32_project(Wo)"); return PSA_ERR_CUDA; }
         return PSA_OK;
     }
-    return bf16_project(y, Ws, outs, 1, batch * n, heads * d_k, d_model, cx.last_dc, stream);
+    return bf16_project(y, Ws, outs, 1, batch * n, heads * d_k, d_model, R, cx.last_dc, stream);
 }
 
 size_t psa_block_workspace_bytes(int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype) {

@@ -65,7 +65,7 @@ struct PMaps {
 struct PBars {
     uint64_t item_full[2], item_empty[2];
     uint64_t q_full[2], q_empty[2];
-    uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
+    uint64_t k_full[8], k_empty[8], v_full[4], v_empty[4];
     uint64_t s_full[2], s_free[2], p_ready[2], o_done[2];
 };
 
@@ -90,18 +90,22 @@ constexpr int ISSUER1_WARP = CTRL_WARPS + 2 * SOFTMAX_WARPS_PER_TILE;
 template <int D> __host__ __device__ constexpr int persist_threads() { return ATTN_THREADS + (D == 64 ? 32 : 0); }
 template <int D> __host__ __device__ constexpr int item_readers() { return (D == 64 ? 2 : 1) + 2 * SOFTMAX_WARPS_PER_TILE; }   // issuers + one lane per softmax warp
 
-template <int D>
+// KVS ("keys are the values"): K and V are one tensor (the case the paper mentions in Sec. 3.1 beside query = key =
+// value).  A key tile is then loaded once and serves phase 1 as the K-major operand and phase 3 as the MN-major
+// one; the shared-memory stages of the V ring extend the K ring, and a tile is released behind its PV.
+template <int D, bool KVS>
 __global__ void __launch_bounds__(persist_threads<D>(), 1)
 attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ SchedParams sp, int H, int scheme,
                     int nitems, float sl2, DeviceCounters* dc, DeviceCounters* dc_next) {
     using Cfg = PCfg<D>;
     constexpr bool SEP = Cfg::SEP_P;
-    constexpr int KST = Cfg::KSTAGES, VST = Cfg::VSTAGES;
+    constexpr int VST = Cfg::VSTAGES;
+    constexpr int KST = KVS ? Cfg::KSTAGES + Cfg::VSTAGES : Cfg::KSTAGES;     // stages of the K ring
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;                                          // 2 tiles
     uint8_t* sK = sQ + 2 * Cfg::TILE_BYTES;                      // KSTAGES tiles
-    uint8_t* sV = sK + KST * Cfg::TILE_BYTES;                    // VSTAGES tiles
+    uint8_t* sV = sK + Cfg::KSTAGES * Cfg::TILE_BYTES;           // VSTAGES tiles (KVS: stages KSTAGES.. of the K ring)
     uint8_t* sStage = sV + VST * Cfg::TILE_BYTES;                // STAGE_BUFS output staging tiles
     __shared__ PBars bars;
     __shared__ uint32_t tmem_base_s;
@@ -133,11 +137,11 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
             mbar_init(&bars.p_ready[t], 32 * SOFTMAX_WARPS_PER_TILE);
             mbar_init(&bars.o_done[t], 1);
         }
-        for (int s = 0; s < 4; ++s) {
+        for (int s = 0; s < 8; ++s) {
             // (with an issuer per slot, an operand tile collects one release from each of them)
             mbar_init(&bars.k_full[s], 1); mbar_init(&bars.k_empty[s], SEP ? 2 : 1);
-            mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], SEP ? 2 : 1);
         }
+        for (int s = 0; s < 4; ++s) { mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], SEP ? 2 : 1); }
         fence_mbar_init();
     }
     if (warp == 1) { tmem_alloc(&tmem_base_s, 512); tmem_relinquish(); }
@@ -192,7 +196,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                         }
                         if (!ok) break;
                     }
-                    {
+                    if constexpr (!KVS) {
                         const int s = vc % VST;
                         if (vc >= (uint32_t)VST) ok = mbar_wait(&bars.v_empty[s], ((vc / VST) - 1) & 1, abortp);
                         if (!ok) break;
@@ -226,7 +230,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
             unsigned long long qk_blocks = 0, pv_blocks = 0;
             const uint32_t q_lo = umma_desc_lo_kmajor(smem_u32(sQ + t * Cfg::TILE_BYTES));
             const uint32_t k_lo = umma_desc_lo_kmajor(smem_u32(sK));
-            const uint32_t v_lo = umma_desc_lo_mnmajor(smem_u32(sV), 16384);
+            const uint32_t v_lo = umma_desc_lo_mnmajor(smem_u32(KVS ? sK : sV), 16384);     // KVS: V_j is the tile of K_j
             const uint32_t dS = tmem + Cfg::TMEM_S + t * 128, dO = tmem + Cfg::TMEM_O + t * D;
             const uint32_t aP = tmem + Cfg::TMEM_P + t * 64;
             uint32_t kbase = 0, vbase = 0;      // ring positions of the current item's first K and V tile
@@ -244,7 +248,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                 ++qk_blocks;
             };
             auto mma_PV = [&](uint32_t vc, bool first) {   // O (+)= P V with V at ring position vc (phase 3, Eq. 3)
-                const uint32_t v = v_lo + (vc % VST) * (Cfg::TILE_BYTES >> 4);
+                const uint32_t v = v_lo + (vc % (KVS ? KST : VST)) * (Cfg::TILE_BYTES >> 4);
                 if (first) {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
@@ -280,7 +284,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                     tc_fence_after();
                     mma_S(kbase);
                     umma_commit(&bars.s_full[t]);
-                    release(&bars.k_empty[kbase % KST], 0 >= nkv_other);
+                    if constexpr (!KVS) release(&bars.k_empty[kbase % KST], 0 >= nkv_other);
                     if (nkv == 1) umma_commit(&bars.q_empty[t]);
                     for (int j = 0; j < nkv && ok; ++j) {
                         const uint32_t vc = vbase + j, kc = kbase + j + 1;
@@ -292,16 +296,17 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                             tc_fence_after();
                             mma_S(kc);
                             umma_commit(&bars.s_full[t]);
-                            release(&bars.k_empty[kc % KST], j + 1 >= nkv_other);
+                            if constexpr (!KVS) release(&bars.k_empty[kc % KST], j + 1 >= nkv_other);
                             if (j + 1 == nkv - 1) umma_commit(&bars.q_empty[t]);
                         }
-                        ok = mbar_wait(&bars.v_full[vc % VST], (vc / VST) & 1, abortp) &&
-                             mbar_wait(&bars.p_ready[t], (blk0 + j) & 1, abortp);
+                        if constexpr (!KVS) ok = mbar_wait(&bars.v_full[vc % VST], (vc / VST) & 1, abortp);
+                        if (ok) ok = mbar_wait(&bars.p_ready[t], (blk0 + j) & 1, abortp);
                         if (!ok) break;
                         tc_fence_after();
-                        mma_PV(vc, j == 0);
+                        mma_PV(KVS ? kbase + j : vc, j == 0);
                         umma_commit(&bars.o_done[t]);
-                        release(&bars.v_empty[vc % VST], j >= nkv_other);
+                        if constexpr (KVS) release(&bars.k_empty[(kbase + j) % KST], j >= nkv_other);    // the tile's last use
+                        else release(&bars.v_empty[vc % VST], j >= nkv_other);
                     }
                     ++parts;
                     blk0 += nkv;
@@ -329,7 +334,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
             unsigned long long qk_blocks = 0, pv_blocks = 0;
             const uint32_t q_lo[2] = {umma_desc_lo_kmajor(smem_u32(sQ)), umma_desc_lo_kmajor(smem_u32(sQ + Cfg::TILE_BYTES))};
             const uint32_t k_lo = umma_desc_lo_kmajor(smem_u32(sK));
-            const uint32_t v_lo = umma_desc_lo_mnmajor(smem_u32(sV), 16384);
+            const uint32_t v_lo = umma_desc_lo_mnmajor(smem_u32(KVS ? sK : sV), 16384);     // KVS: V_j is the tile of K_j
             const uint32_t tS0 = tmem + Cfg::TMEM_S, tO0 = tmem + Cfg::TMEM_O;
             uint32_t kbase = 0, vbase = 0;      // ring positions of the current item's first K and V tile
             uint32_t parts[2] = {0, 0};         // earlier items in which tile slot t had rows
@@ -349,7 +354,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
             };
             // O_t (+)= P_t V with V at ring position vc (phase 3, Eq. 3): 8 MMAs of 128 x D x 16.
             auto mma_PV = [&](int t, uint32_t vc, bool first) {
-                const uint32_t v = v_lo + (vc % VST) * (Cfg::TILE_BYTES >> 4);
+                const uint32_t v = v_lo + (vc % (KVS ? KST : VST)) * (Cfg::TILE_BYTES >> 4);
                 const uint32_t dO = tO0 + t * D;
                 const uint32_t aP = SEP ? tmem + Cfg::TMEM_P + t * 64 : tS0 + t * 128;
                 if (first) {
@@ -387,26 +392,27 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                         if (nkv[t] == 1) umma_commit(&bars.q_empty[t]);
                     }
                     if (!ok) break;
-                    umma_commit(&bars.k_empty[kbase % KST]);
+                    if constexpr (!KVS) umma_commit(&bars.k_empty[kbase % KST]);
                     for (int j = 0; j < maxkv && ok; ++j) {
                         for (int t = 0; t < work.ntiles && ok; ++t) {
                             if (j >= nkv[t]) continue;
                             const uint32_t vc = vbase + j, kc = kbase + j + 1;
                             const bool has_next = j + 1 < nkv[t];
                             // operand tiles first: these are normally long complete and cost only the poll
-                            ok = mbar_wait(&bars.v_full[vc % VST], (vc / VST) & 1, abortp);
+                            if constexpr (!KVS) ok = mbar_wait(&bars.v_full[vc % VST], (vc / VST) & 1, abortp);
                             if (ok && has_next) ok = mbar_wait(&bars.k_full[kc % KST], (kc / KST) & 1, abortp);
                             if (ok) ok = mbar_wait(&bars.p_ready[t], (blk0[t] + j) & 1, abortp);
                             if (!ok) break;
                             tc_fence_after();
-                            mma_PV(t, vc, j == 0);
+                            mma_PV(t, KVS ? kbase + j : vc, j == 0);
                             if (has_next) mma_S(t, kc);
                             umma_commit(&bars.o_done[t]);
                             // an operand tile is released behind its last user in this fixed order
                             const bool last_v = t == work.ntiles - 1 || j >= nkv[t + 1];
-                            if (last_v) umma_commit(&bars.v_empty[vc % VST]);
+                            if (last_v) umma_commit(KVS ? &bars.k_empty[(kbase + j) % KST] : &bars.v_empty[vc % VST]);
                             if (has_next) {
-                                if (t == work.ntiles - 1 || j + 1 >= nkv[t + 1]) umma_commit(&bars.k_empty[kc % KST]);
+                                if constexpr (!KVS)
+                                    if (t == work.ntiles - 1 || j + 1 >= nkv[t + 1]) umma_commit(&bars.k_empty[kc % KST]);
                                 if (j + 1 == nkv[t] - 1) umma_commit(&bars.q_empty[t]);
                             }
                         }
@@ -615,13 +621,13 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
-template <int D>
+template <int D, bool KVS>
 int launch_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, float scale,
                    int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream) {
     using Cfg = PCfg<D>;
     static DeviceSetup setup;
     const int sm_count = device_setup(&setup, [] {
-        return cudaFuncSetAttribute(attn_persist_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, PCfg<D>::SMEM);
+        return cudaFuncSetAttribute(attn_persist_kernel<D, KVS>, cudaFuncAttributeMaxDynamicSharedMemorySize, PCfg<D>::SMEM);
     }, "attention kernel set-up");
     if (sm_count <= 0) return PSA_ERR_CUDA;
     const uint64_t cols = (uint64_t)H * D;
@@ -636,7 +642,7 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
     const int grid = (int)(nitems < sm_count ? nitems : sm_count);
     const SchedParams sp = sched_params(n, scheme == PSA_MASKED, B * H, lpt_group(scheme, B * H, n, D),
                                         split == pairs ? 0x7fffffff : (int)split);
-    attn_persist_kernel<D><<<grid, persist_threads<D>(), Cfg::SMEM, stream>>>(maps, sp, H, scheme, (int)nitems,
+    attn_persist_kernel<D, KVS><<<grid, persist_threads<D>(), Cfg::SMEM, stream>>>(maps, sp, H, scheme, (int)nitems,
                                                                             scale * LOG2E, dc, dc_next);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "attn_persist_kernel launch"); return PSA_ERR_CUDA; }
@@ -650,8 +656,13 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
 int bf16_attention_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, int d,
                            float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream) {
     if (scheme != PSA_FULL && scheme != PSA_MASKED) return PSA_ERR_SCHEME_ARGS;
-    if (d == 64) return launch_persist<64>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
-    if (d == 128) return launch_persist<128>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
+    if (K == V) {     // one tensor for keys and values: each key tile is loaded once
+        if (d == 64) return launch_persist<64, true>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
+        if (d == 128) return launch_persist<128, true>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
+        return PSA_ERR_UNSUPPORTED;
+    }
+    if (d == 64) return launch_persist<64, false>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
+    if (d == 128) return launch_persist<128, false>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
     return PSA_ERR_UNSUPPORTED;
 }
 

@@ -13,7 +13,7 @@ constexpr int PROJ_TILE = 16;
 // out[w][r, c] = sum_k X[r, k] W[w][k, c]      (paper Sec. 3.1: the projections are plain products)
 __global__ void __launch_bounds__(PROJ_TILE* PROJ_TILE)
 f32_project_kernel(const float* __restrict__ X, const float* W0, const float* W1, const float* W2, float* O0,
-                   float* O1, float* O2, int rows, int D, int N, DeviceCounters* dc) {
+                   float* O1, float* O2, int rows, int D, int N, const float* __restrict__ R, DeviceCounters* dc) {
     __shared__ float xs[PROJ_TILE][PROJ_TILE + 1];
     __shared__ float ws[PROJ_TILE][PROJ_TILE + 1];
     const float* W = blockIdx.z == 0 ? W0 : (blockIdx.z == 1 ? W1 : W2);
@@ -29,7 +29,7 @@ f32_project_kernel(const float* __restrict__ X, const float* W0, const float* W1
         for (int k = 0; k < PROJ_TILE; ++k) acc = fmaf(xs[ty][k], ws[k][tx], acc);
         __syncthreads();
     }
-    if (r < rows && c < N) O[(size_t)r * N + c] = acc;
+    if (r < rows && c < N) O[(size_t)r * N + c] = R ? acc + R[(size_t)r * N + c] : acc;
     if (tx == 0 && ty == 0) {
         const int vr = min(PROJ_TILE, rows - blockIdx.y * PROJ_TILE), vc = min(PROJ_TILE, N - blockIdx.x * PROJ_TILE);
         atomicAdd(&dc->proj_macs, (unsigned long long)vr * vc * D);
@@ -143,9 +143,9 @@ size_t attn_smem_bytes(int n, int d) {
 }  // namespace
 
 cudaError_t f32_project(const float* X, const float* const W[3], float* const out[3], int nW, int rows, int D,
-                        int N, DeviceCounters* dc, cudaStream_t stream) {
+                        int N, const float* residual, DeviceCounters* dc, cudaStream_t stream) {
     dim3 block(PROJ_TILE, PROJ_TILE), grid((N + PROJ_TILE - 1) / PROJ_TILE, (rows + PROJ_TILE - 1) / PROJ_TILE, nW);
-    f32_project_kernel<<<grid, block, 0, stream>>>(X, W[0], W[1], W[2], out[0], out[1], out[2], rows, D, N, dc);
+    f32_project_kernel<<<grid, block, 0, stream>>>(X, W[0], W[1], W[2], out[0], out[1], out[2], rows, D, N, residual, dc);
     return cudaGetLastError();
 }
 

@@ -1,5 +1,6 @@
 // Projection GEMM for the bf16 path (paper Sec. 3.1: q, k, v = x*Wq, x*Wk, x*Wv):
-//     C_w[M, N] = A[M, K] * B_w[K, N],  w < nW,  bf16 row-major operands, fp32 accumulation in TMEM.
+//     C_w[M, N] = A[M, K] * B_w[K, N] (+ R[M, N]),  w < nW,  bf16 row-major operands, fp32 accumulation in TMEM;
+// the optional residual R is added in the epilogue (the output projection of the attention block).
 //
 // Persistent kernel, one CTA per SM, walking 128 x 256 output tiles (all three weight matrices in one
 // launch).  Warp 0 streams operand tiles with TMA into a shared-memory ring, warp 1 issues tcgen05 MMAs
@@ -116,7 +117,8 @@ __device__ __forceinline__ TileCoord tile_coord(int t, int mt, int nt) {
 }
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, int nW, DeviceCounters* dc) {
+gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, int nW, const uint16_t* __restrict__ R,
+                 DeviceCounters* dc) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* stage_out = smem + STAGES * STAGE_BYTES;
@@ -229,6 +231,24 @@ gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, int
                 tmem_ld32(src, r[0]);
                 tmem_ld32(src + 32, r[1]);
                 tc_wait_ld();
+                if (R) {
+                    // residual input: C = A B + R, added in fp32 before the rounding to bf16 (R is [M, N] bf16, row-major)
+                    const int grow = c.m0 + row, gcol = c.n0 + 64 * u;
+                    if (grow < M && gcol < N) {
+                        const uint4* rp = reinterpret_cast<const uint4*>(R + (size_t)grow * N + gcol);
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const uint4 x = __ldg(rp + g);
+                            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                uint32_t* dst = &r[g >> 2][(g & 3) * 8 + 2 * e];
+                                dst[0] = __float_as_uint(__uint_as_float(dst[0]) + __uint_as_float(w[e] << 16));
+                                dst[1] = __float_as_uint(__uint_as_float(dst[1]) + __uint_as_float(w[e] & 0xffff0000u));
+                            }
+                        }
+                    }
+                }
 #pragma unroll
                 for (int c0 = 0; c0 < 2; ++c0) {
 #pragma unroll
@@ -267,7 +287,7 @@ gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, int
 }  // namespace
 
 int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int nW, int M, int K, int N,
-                 DeviceCounters* dc, cudaStream_t stream) {
+                 const void* residual, DeviceCounters* dc, cudaStream_t stream) {
     static DeviceSetup setup;
     const int sm_count = device_setup(&setup, [] {
         return cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
@@ -282,7 +302,7 @@ int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int n
     }
     const int ntiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN) * nW;
     const int grid = ntiles < sm_count ? ntiles : sm_count;
-    gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(maps, M, N, K, nW, dc);
+    gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(maps, M, N, K, nW, static_cast<const uint16_t*>(residual), dc);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error(e, "gemm_bf16_kernel launch"); return PSA_ERR_CUDA; }
     return PSA_OK;

@@ -23,16 +23,18 @@ struct DeviceCounters {
 
 // ---- fp32 CUDA-core path (psa_f32.cu) ----
 // out[w][r, c] = sum_k X[r, k] W[w][k, c] for w < nW.
+// `residual` ([rows, N], may be null) is added to every output.
 cudaError_t f32_project(const float* X, const float* const W[3], float* const out[3], int nW, int rows, int D,
-                        int N, DeviceCounters* dc, cudaStream_t stream);
+                        int N, const float* residual, DeviceCounters* dc, cudaStream_t stream);
 // Q, K, V, out: [B, n, H, d] fp32.  S: scratch [B*H, n, n] fp32, used by PSA_SYMMETRIC only.
 cudaError_t f32_attention(const float* Q, const float* K, const float* V, float* out, float* S, int B, int H,
                           int n, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
 
 // ---- bf16 tcgen05 path (psa_gemm.cu, psa_attn.cu) ----
-// C[w][M, N] = A[M, K] * Bw[w][K, N], bf16 row-major, fp32 accumulation.  Returns a psa_status.
+// C[w][M, N] = A[M, K] * Bw[w][K, N] (+ residual[M, N], bf16, may be null), bf16 row-major, fp32 accumulation.
+// Returns a psa_status.
 int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int nW, int M, int K, int N,
-                 DeviceCounters* dc, cudaStream_t stream);
+                 const void* residual, DeviceCounters* dc, cudaStream_t stream);
 // Q, K, V, out: [B, n, H, d] bf16.  S: scratch for PSA_SYMMETRIC (bf16_symmetric_scratch_bytes:
 // one 64 KB fp32 image per score block at or below the block diagonal, for the heads of one pass).
 // `dc_next`, if not null, is a second counter block that the call's attention kernel clears (FULL, MASKED only).

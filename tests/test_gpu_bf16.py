@@ -178,3 +178,22 @@ def test_core_host_entry_matches_device_entry():
         out_d = binding.psa_attention_core(host[0].cuda(), None if sym else host[1].cuda(),
                                            None if sym else host[2].cuda(), scheme)
         assert torch.equal(out_h.view(torch.int16), out_d.cpu().view(torch.int16))
+
+
+@pytest.mark.parametrize("scheme", [oracle.FULL, oracle.MASKED])
+@pytest.mark.parametrize("B,H,n,d", [(1, 1, 128, 64), (1, 2, 640, 128), (2, 3, 384, 64), (2, 2, 1000, 128), (1, 2, 333, 64),
+                                     (3, 100, 256, 128), (4, 40, 384, 64), (1, 1, 2048, 128), (1, 2, 1536, 64)])
+def test_keys_equal_values(scheme, B, H, n, d):
+    # One tensor serves as keys and values (K = V != Q, the case Sec. 3.1 mentions): the kernel loads each key tile
+    # once and uses it in both phases.  Same values and census as with two equal tensors.
+    qv, qb = inputs.tensor(41 * n + d, 4, (B, n, H, d), 1.0, "bf16")
+    kv, kb = inputs.tensor(41 * n + d, 5, (B, n, H, d), 1.0, "bf16")
+    q, k = _dev_bf16(qb), _dev_bf16(kb)
+    out = binding.psa_attention_core(q, k, k, scheme)
+    _check_census(B, H, n, 0, d, scheme)
+    if B * H * n * n <= 3 * 1024 * 1024:
+        ref, _ = oracle.attention_core(qv, kv, kv, scheme)
+        assert np.abs(_to_f64(out) - ref).max() <= TOL_BF16
+    # two distinct tensors with the same contents take the two-ring path: bitwise the same result
+    out2 = binding.psa_attention_core(q, k, k.clone(), scheme)
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16))

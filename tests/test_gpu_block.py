@@ -105,3 +105,51 @@ def test_block_workspace_and_argument_errors():
     sym = (B, H, n, D, d, int(oracle.SYMMETRIC), binding.BF16, p(x), None)
     w2 = torch.zeros_like(w)
     assert L.psa_attention_block(p(x), p(w), p(w2), None, p(w), *sym) == binding.ERR_SCHEME_ARGS
+
+
+@pytest.mark.parametrize("scheme", [oracle.FULL, oracle.MASKED, oracle.SYMMETRIC])
+@pytest.mark.parametrize("B,H,n,D,d", [(1, 1, 128, 64, 64), (2, 3, 256, 192, 64), (2, 2, 333, 128, 64), (1, 2, 384, 320, 128)])
+def test_block_with_residual_bf16_matches_oracle(scheme, B, H, n, D, d):
+    # z = R + y Wo with R = X (the usual skip connection) and with an unrelated R; the sum is formed in fp32 before
+    # the rounding of z, so the tolerance is that of the block
+    sym = scheme == oracle.SYMMETRIC
+    Xv, Xb = inputs.tensor(21, 0, (B, n, D), 1.0, "bf16")
+    W = [inputs.tensor(21, 1 + i, (D, H * d), D ** -0.5, "bf16") for i in range(3)]
+    Wov, Wob = inputs.tensor(21, 8, (H * d, D), (H * d) ** -0.5, "bf16")
+    Rv, Rb = inputs.tensor(21, 9, (B, n, D), 2.0, "bf16")
+    X = _dev_bf16(Xb)
+    for res_v, res_dev in ((Xv, X), (Rv, _dev_bf16(Rb))):
+        out = binding.psa_attention_block(X, _dev_bf16(W[0][1]), None if sym else _dev_bf16(W[1][1]),
+                                          None if sym else _dev_bf16(W[2][1]), _dev_bf16(Wob), H, scheme, residual=res_dev)
+        ref, _, _ = oracle.attention_block(Xv, W[0][0], W[1][0], W[2][0], Wov, H, scheme, residual=res_v)
+        excess = (np.abs(_to_f64(out) - ref) - TOL_BF16_REL * np.abs(ref)).max()
+        assert excess <= TOL_BF16, excess
+        st, got = binding.psa_last_issued()
+        assert st == binding.OK and got["proj_macs"] == _proj_macs(B, H, n, D, d, scheme)
+
+
+@pytest.mark.parametrize("scheme", [oracle.FULL, oracle.MASKED, oracle.SYMMETRIC])
+def test_block_with_residual_f32_matches_oracle(scheme):
+    B, H, n, D, d = 2, 3, 37, 50, 20
+    rng = np.random.default_rng(77)
+    X = (rng.standard_normal((B, n, D)) * 0.5).astype(np.float32)
+    Ws = [(rng.standard_normal((D, H * d)) / np.sqrt(D)).astype(np.float32) for _ in range(3)]
+    Wo = (rng.standard_normal((H * d, D)) / np.sqrt(H * d)).astype(np.float32)
+    R = rng.standard_normal((B, n, D)).astype(np.float32)
+    sym = scheme == oracle.SYMMETRIC
+    dev = lambda a: torch.from_numpy(a).cuda()
+    out = binding.psa_attention_block(dev(X), dev(Ws[0]), None if sym else dev(Ws[1]), None if sym else dev(Ws[2]),
+                                      dev(Wo), H, scheme, residual=dev(R))
+    ref, _, _ = oracle.attention_block(X, Ws[0], Ws[1], Ws[2], Wo, H, scheme, residual=R)
+    assert np.abs(out.cpu().numpy().astype(np.float64) - ref).max() <= TOL_F32
+
+
+def test_block_residual_must_not_be_the_output():
+    B, H, n, D, d = 1, 2, 128, 128, 64
+    x = torch.zeros((B, n, D), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((D, H * d), dtype=torch.bfloat16, device="cuda")
+    wo = torch.zeros((H * d, D), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros_like(x)
+    with pytest.raises(binding.PsaError) as ei:
+        binding.psa_attention_block(x, w, w, w, wo, H, oracle.FULL, out=out, residual=out)
+    assert ei.value.status == binding.ERR_SCHEME_ARGS
