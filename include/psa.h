@@ -74,8 +74,9 @@ typedef struct {
  * Projections + attention, bf16 in / bf16 out, fp32 accumulation (paper Sec. 3.1 then Eq. 1-3).
  *   X, Wq, Wk, Wv, out   device, bf16, layouts above.
  *   PSA_SYMMETRIC: q = k = v = X*Wq (paper Sec. 4.1); Wk and Wv must be NULL or equal to Wq.
- * Supported: d_k in {64, 128}; any n >= 1 (a last block of fewer than 128 vectors is zero-filled and its
- * keys carry no weight); d_model and heads*d_k multiples of 64.
+ * Supported: d_k any multiple of 8 up to 128 (the kernels work on heads of 64 or 128 columns; a shorter head is
+ * zero-padded by the tile loads, and the census counts the padded width as issued); any n >= 1 (a last block of
+ * fewer than 128 vectors is zero-filled and its keys carry no weight); d_model and heads*d_k multiples of 64.
  * Needs a workspace of psa_workspace_bytes(...) (grown on demand, see psa_set_workspace).
  */
 int psa_attention(const void* X, const void* Wq, const void* Wk, const void* Wv, int batch, int heads, int n,
@@ -90,7 +91,9 @@ int psa_attention_f32(const void* X, const void* Wq, const void* Wk, const void*
  * Attention core only (paper Eq. 1-3 with q, k, v given; Sec. 3.1 last paragraph).
  *   dtype PSA_BF16 or PSA_F32 selects the path and the storage type of Q, K, V, out.
  *   PSA_SYMMETRIC: K and V must be NULL or equal to Q.
- * Shape limits as for psa_attention / psa_attention_f32.
+ *   PSA_FULL / PSA_MASKED with K == V (one tensor for keys and values, paper Sec. 3.1): each key tile is loaded
+ *   once and serves both phases.
+ * Shape limits as for psa_attention / psa_attention_f32 (heads*d_k need not be a multiple of 64 here).
  */
 int psa_attention_core(const void* Q, const void* K, const void* V, int batch, int heads, int n, int d_k,
                        int scheme, int dtype, void* out, void* stream);

@@ -61,7 +61,7 @@ int check_shape(int batch, int heads, int n, int d_model, int d_k, int scheme, i
         return PSA_ERR_SHAPE;
     if ((long long)batch * n > 0x7fffffffLL || (long long)heads * d_k > 0x7fffffffLL) return PSA_ERR_SHAPE;
     if (dtype == PSA_BF16) {
-        if (d_k != 64 && d_k != 128) return PSA_ERR_UNSUPPORTED;
+        if (d_k < 8 || d_k > 128 || d_k % 8 != 0) return PSA_ERR_UNSUPPORTED;
         if (with_proj && (d_model % 64 != 0)) return PSA_ERR_UNSUPPORTED;
     } else {
         if (n > 1024 || d_k > 128) return PSA_ERR_UNSUPPORTED;
@@ -427,7 +427,9 @@ int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme
     // pairs of a launch out as single row tiles, split_point in psa_sched.h, those are the same row tiles with the
     // same block lists taken one at a time: the census does not depend on the grouping.)
     const int T = row_tiles(n);
-    const uint64_t block_macs = (uint64_t)TILE * TILE * d_k;
+    // (a head size below the 64 or 128 columns the kernels work with is zero-padded by the loads: the padded
+    // width is what the tensor core is issued)
+    const uint64_t block_macs = (uint64_t)TILE * TILE * (d_k <= 64 ? 64 : 128);
     uint64_t qk_blocks = 0, pv_blocks = 0, exps = 0;
     const int P = ctas_per_head(n);
     for (int cta = 0; cta < P; ++cta) {  // every head has the same list

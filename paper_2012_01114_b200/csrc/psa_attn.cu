@@ -80,7 +80,6 @@ sym_scores_kernel(const __grid_constant__ SymMaps maps, float* __restrict__ Sg, 
     int I, J;
     sym_pair(blockIdx.x - hl * np, &I, &J);
     const int bh = bh0 + hl, b = bh / H, h = bh - b * H;
-    const int col0 = h * D;
     const int pair = blockIdx.x - hl * np;           // = I (I + 1) / 2 + J: the block's place in the head's scratch
 
     if (threadIdx.x == 0) {
@@ -99,8 +98,8 @@ sym_scores_kernel(const __grid_constant__ SymMaps maps, float* __restrict__ Sg, 
     if (threadIdx.x == 0) {
         mbar_arrive_expect_tx(&full_bar, 2 * TILE_BYTES);
         for (int u = 0; u < SUB; ++u) {
-            tma_load_3d(sA + u * 16384, &maps.x, &full_bar, col0 + 64 * u, I * TILE, b);
-            tma_load_3d(sB + u * 16384, &maps.x, &full_bar, col0 + 64 * u, J * TILE, b);
+            tma_load_4d(sA + u * 16384, &maps.x, &full_bar, 64 * u, h, I * TILE, b);
+            tma_load_4d(sB + u * 16384, &maps.x, &full_bar, 64 * u, h, J * TILE, b);
         }
         if (mbar_wait(&full_bar, 0, abortp)) {
             tc_fence_after();
@@ -183,7 +182,6 @@ sym_attn_kernel(const __grid_constant__ SymMaps maps, const float* __restrict__ 
     const int It = blockIdx.x - hl * T;                  // row tile
     const int bh = bh0 + hl;
     const int b = bh / H, h = bh - b * H;
-    const int col0 = h * D;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -225,7 +223,7 @@ sym_attn_kernel(const __grid_constant__ SymMaps maps, const float* __restrict__ 
                 if (!ok) break;
                 mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
                 for (int u = 0; u < Cfg::SUB; ++u)
-                    tma_load_3d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.x, &bars.v_full[s], col0 + 64 * u, j * TILE, b);
+                    tma_load_4d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.x, &bars.v_full[s], 64 * u, h, j * TILE, b);
                 ++v_loads;
             }
             if (*abortp) {  // let copies already issued land before shared memory is released
@@ -398,7 +396,7 @@ sym_attn_kernel(const __grid_constant__ SymMaps maps, const float* __restrict__ 
             named_bar_sync(tile_bar, 32 * SOFTMAX_WARPS_PER_TILE);
             if (sw == 0 && lane == 0) {
                 for (int u = 0; u < Cfg::SUB; ++u)
-                    tma_store_3d(&maps.o, stage + u * 16384, col0 + 64 * u, It * TILE, b);
+                    tma_store_4d(&maps.o, stage + u * 16384, 64 * u, h, It * TILE, b);
                 tma_store_commit();
                 tma_store_wait_read();   // smem may be released; the writes complete on their own
             }
@@ -424,8 +422,9 @@ int sym_heads_per_pass(int B, int H, int n) {
     return (int)((all + passes - 1) / passes);
 }
 
+// D: head size the kernels work with (64 or 128); d <= D: the tensors' head size (see the 4-D tensor maps).
 template <int D>
-int launch_symmetric(const void* X, void* out, float* S, int B, int H, int n, float scale, DeviceCounters* dc,
+int launch_symmetric(const void* X, void* out, float* S, int B, int H, int n, int d, float scale, DeviceCounters* dc,
                      cudaStream_t stream) {
     using Cfg = SymCfg<D>;
     static DeviceSetup setup;
@@ -438,9 +437,8 @@ int launch_symmetric(const void* X, void* out, float* S, int B, int H, int n, fl
         return PSA_ERR_CUDA;
     const int T = row_tiles(n), np = sym_pairs(T);
     const int hp = sym_heads_per_pass(B, H, n);
-    const uint64_t cols = (uint64_t)H * D;
     SymMaps maps;
-    if (!make_tensor_map_bf16_3d(&maps.x, X, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.o, out, B, n, cols, 128))
+    if (!make_tensor_map_bf16_4d(&maps.x, X, B, n, H, d, 128) || !make_tensor_map_bf16_4d(&maps.o, out, B, n, H, d, 128))
         return PSA_ERR_CUDA;
     for (int bh0 = 0; bh0 < B * H; bh0 += hp) {
         const int heads = min(hp, B * H - bh0);
@@ -465,9 +463,9 @@ int bf16_attention(const void* Q, const void* K, const void* V, void* out, float
     if (scheme != PSA_SYMMETRIC) return bf16_attention_persist(Q, K, V, out, B, H, n, d, scale, scheme, dc, dc_next, stream);
     if (!S || s_bytes < bf16_symmetric_scratch_bytes(B, H, n)) return PSA_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(S) & 15u) != 0) return PSA_ERR_ALIGN;
-    if (d == 64) return launch_symmetric<64>(Q, out, S, B, H, n, scale, dc, stream);
-    if (d == 128) return launch_symmetric<128>(Q, out, S, B, H, n, scale, dc, stream);
-    return PSA_ERR_UNSUPPORTED;
+    if (d < 8 || d > 128 || d % 8) return PSA_ERR_UNSUPPORTED;
+    if (d <= 64) return launch_symmetric<64>(Q, out, S, B, H, n, d, scale, dc, stream);
+    return launch_symmetric<128>(Q, out, S, B, H, n, d, scale, dc, stream);
 }
 
 }  // namespace psa

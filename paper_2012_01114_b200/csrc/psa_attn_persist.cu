@@ -169,7 +169,6 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                 // the next item's index is fetched now, long before it is needed
                 const int next = (int)gridDim.x + (int)atomicAdd(&dc->next_item, 1u);
                 const int b = work.bh / H, h = work.bh - b * H;
-                const int col0 = h * D;
                 const int nkv0 = kv_tiles(work.tile0, T, scheme);
                 const int nkv1 = work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0;
                 const int maxkv = max(nkv0, nkv1);
@@ -180,7 +179,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                         if (!ok) break;
                         mbar_arrive_expect_tx(&bars.k_full[s], Cfg::TILE_BYTES);
                         for (int u = 0; u < Cfg::SUB; ++u)
-                            tma_load_3d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], col0 + 64 * u,
+                            tma_load_4d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], 64 * u, h,
                                         j * TILE, b);
                         ++kc;
                     }
@@ -190,8 +189,8 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                             if (!ok) break;
                             mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
                             for (int u = 0; u < Cfg::SUB; ++u)
-                                tma_load_3d(sQ + t * Cfg::TILE_BYTES + u * 16384, &maps.q, &bars.q_full[t],
-                                            col0 + 64 * u, (work.tile0 + t) * TILE, b);
+                                tma_load_4d(sQ + t * Cfg::TILE_BYTES + u * 16384, &maps.q, &bars.q_full[t],
+                                            64 * u, h, (work.tile0 + t) * TILE, b);
                             ++qc[t];
                         }
                         if (!ok) break;
@@ -202,7 +201,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                         if (!ok) break;
                         mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
                         for (int u = 0; u < Cfg::SUB; ++u)
-                            tma_load_3d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], col0 + 64 * u,
+                            tma_load_4d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], 64 * u, h,
                                         j * TILE, b);
                         ++vc;
                     }
@@ -599,10 +598,10 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
             else ok = named_bar_all(ok, pair_bar, 32 * TPR);
             if (ok && (Cfg::WARP_UNITS || part == 0) && lane == 0) {
                 if (Cfg::WARP_UNITS) {
-                    tma_store_3d(&maps.o, stage, h * D + part * OPT, It * TILE + q * 32, b);
+                    tma_store_4d(&maps.o, stage, part * OPT, h, It * TILE + q * 32, b);
                 } else {
                     for (int u = 0; u < Cfg::SUB; ++u)
-                        tma_store_3d(&maps.o, stage + u * 4096, h * D + 64 * u, It * TILE + q * 32, b);
+                        tma_store_4d(&maps.o, stage + u * 4096, 64 * u, h, It * TILE + q * 32, b);
                 }
                 tma_store_commit();
                 tma_store_wait_read();   // the buffer may be rewritten; the global writes complete on their own
@@ -621,8 +620,10 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
+// D: head size the kernel works with (64 or 128); d: the tensors' head size, d <= D, a multiple of 8 (the columns
+// between d and D are zero-filled by the loads and dropped by the stores).
 template <int D, bool KVS>
-int launch_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, float scale,
+int launch_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, int d, float scale,
                    int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream) {
     using Cfg = PCfg<D>;
     static DeviceSetup setup;
@@ -630,17 +631,16 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
         return cudaFuncSetAttribute(attn_persist_kernel<D, KVS>, cudaFuncAttributeMaxDynamicSharedMemorySize, PCfg<D>::SMEM);
     }, "attention kernel set-up");
     if (sm_count <= 0) return PSA_ERR_CUDA;
-    const uint64_t cols = (uint64_t)H * D;
     PMaps maps;
-    if (!make_tensor_map_bf16_3d(&maps.q, Q, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.k, K, B, n, cols, 128) ||
-        !make_tensor_map_bf16_3d(&maps.v, V, B, n, cols, 128) || !make_tensor_map_bf16_3d(&maps.o, out, B, n, cols, 32))
+    if (!make_tensor_map_bf16_4d(&maps.q, Q, B, n, H, d, 128) || !make_tensor_map_bf16_4d(&maps.k, K, B, n, H, d, 128) ||
+        !make_tensor_map_bf16_4d(&maps.v, V, B, n, H, d, 128) || !make_tensor_map_bf16_4d(&maps.o, out, B, n, H, d, 32))
         return PSA_ERR_CUDA;
     const long long pairs = (long long)B * H * ctas_per_head(n);
     const long long split = D == 64 ? split_point(scheme, pairs, n, sm_count) : pairs;
     const long long nitems = pairs + (pairs - split);          // pairs, then the rest as single row tiles
     if (nitems > 0x7fffffffLL - sm_count) return PSA_ERR_SHAPE;
     const int grid = (int)(nitems < sm_count ? nitems : sm_count);
-    const SchedParams sp = sched_params(n, scheme == PSA_MASKED, B * H, lpt_group(scheme, B * H, n, D),
+    const SchedParams sp = sched_params(n, scheme == PSA_MASKED, B * H, lpt_group(scheme, B * H, n, d),
                                         split == pairs ? 0x7fffffff : (int)split);
     attn_persist_kernel<D, KVS><<<grid, persist_threads<D>(), Cfg::SMEM, stream>>>(maps, sp, H, scheme, (int)nitems,
                                                                             scale * LOG2E, dc, dc_next);
@@ -656,14 +656,13 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
 int bf16_attention_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, int d,
                            float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream) {
     if (scheme != PSA_FULL && scheme != PSA_MASKED) return PSA_ERR_SCHEME_ARGS;
+    if (d < 8 || d > 128 || d % 8) return PSA_ERR_UNSUPPORTED;
     if (K == V) {     // one tensor for keys and values: each key tile is loaded once
-        if (d == 64) return launch_persist<64, true>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
-        if (d == 128) return launch_persist<128, true>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
-        return PSA_ERR_UNSUPPORTED;
+        if (d <= 64) return launch_persist<64, true>(Q, K, V, out, B, H, n, d, scale, scheme, dc, dc_next, stream);
+        return launch_persist<128, true>(Q, K, V, out, B, H, n, d, scale, scheme, dc, dc_next, stream);
     }
-    if (d == 64) return launch_persist<64, false>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
-    if (d == 128) return launch_persist<128, false>(Q, K, V, out, B, H, n, scale, scheme, dc, dc_next, stream);
-    return PSA_ERR_UNSUPPORTED;
+    if (d <= 64) return launch_persist<64, false>(Q, K, V, out, B, H, n, d, scale, scheme, dc, dc_next, stream);
+    return launch_persist<128, false>(Q, K, V, out, B, H, n, d, scale, scheme, dc, dc_next, stream);
 }
 
 }  // namespace psa

@@ -79,6 +79,25 @@ bool make_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t batch,
     return true;
 }
 
+bool make_tensor_map_bf16_4d(CUtensorMap* map, const void* base, uint64_t batch, uint64_t n, uint64_t heads, uint64_t d,
+                             uint32_t box_rows) {
+    if (!resolve_encode()) return false;
+    cuuint64_t dims[4] = {d, heads, n, batch};
+    cuuint64_t strides[3] = {d * 2, heads * d * 2, n * heads * d * 2};
+    cuuint32_t box[4] = {64, 1, box_rows, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char msg[96];
+        snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled (4-D) failed with CUresult %d", (int)r);
+        set_error_text(msg);
+        return false;
+    }
+    return true;
+}
+
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;

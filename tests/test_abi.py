@@ -75,7 +75,10 @@ def test_argument_errors_launch_nothing(lib):
     assert lib.psa_skip_count(1, 1, 128, 0, 64, 7, binding.BF16, ctypes.byref(c)) == binding.ERR_SCHEME_ARGS
     assert lib.psa_skip_count(1, 1, 100, 0, 64, 0, binding.BF16, ctypes.byref(c)) == binding.OK      # ragged n is fine
     assert lib.psa_skip_count(1, 1, 128, 100, 64, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED  # d_model % 64
-    assert lib.psa_skip_count(1, 1, 128, 0, 96, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED
+    assert lib.psa_skip_count(1, 1, 128, 0, 100, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED   # d_k % 8
+    assert lib.psa_skip_count(1, 1, 128, 0, 256, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED   # d_k > 128
+    assert lib.psa_skip_count(1, 1, 128, 0, 96, 0, binding.BF16, ctypes.byref(c)) == binding.OK
+    assert c.qk_macs == 128 * 128 * 128 and c.useful_qk_macs == 128 * 128 * 96    # issued at the padded width of 128
     assert lib.psa_skip_count(1, 1, 2048, 0, 64, 0, binding.F32, ctypes.byref(c)) == binding.ERR_UNSUPPORTED
     assert lib.psa_skip_count(0, 1, 128, 0, 64, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_SHAPE
     assert lib.psa_skip_count(1, 1, 128, 0, 64, 0, binding.BF16, None) == binding.ERR_NULL
@@ -85,6 +88,6 @@ def test_argument_errors_launch_nothing(lib):
     assert lib.psa_attention_core(8, 16, 16, 1, 1, 128, 64, 0, binding.BF16, 16, None) == binding.ERR_ALIGN
     assert lib.psa_attention_core(16, 32, 16, 1, 1, 128, 64, 1, binding.BF16, 16, None) == binding.ERR_SCHEME_ARGS
     assert lib.psa_attention(16, 16, 32, 16, 1, 1, 128, 64, 64, 1, 16, None) == binding.ERR_SCHEME_ARGS
-    assert lib.psa_workspace_bytes(1, 1, 100, 0, 96, 0, binding.BF16, 0) == 0
+    assert lib.psa_workspace_bytes(1, 1, 100, 0, 100, 0, binding.BF16, 0) == 0
     assert binding.psa_status_string(binding.ERR_TIMEOUT).startswith("a bounded")
     assert binding.psa_workspace_bytes(8, 12, 1024, 768, 64, oracle.MASKED, binding.BF16) >= 3 * 8 * 1024 * 768 * 2
