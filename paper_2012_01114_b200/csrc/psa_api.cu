@@ -158,6 +158,15 @@ int run_layer(Context& cx, const void* X, const void* Wq, const void* Wk, const 
         ~EventTail() { if (ev) cudaEventRecord(ev[2], st); }
     } tail{pev, stream};
     if (pev) cudaEventRecord(pev[0], stream);
+    if (with_proj && dtype == PSA_F32 && f32_fused_fits(n, d_model, d_k, scheme)) {
+        // a small fp32 layer runs as one launch; q, k, v never leave shared memory
+        if (pev) cudaEventRecord(pev[1], stream);
+        e = f32_fused_layer(static_cast<const float*>(X), static_cast<const float*>(Wq), static_cast<const float*>(Wk),
+                            static_cast<const float*>(Wv), static_cast<float*>(out), batch, heads, n, d_model, d_k, scale,
+                            scheme, dc, stream);
+        if (e != cudaSuccess) { set_cuda_error(e, "f32_fused_layer"); return PSA_ERR_CUDA; }
+        return PSA_OK;
+    }
     if (with_proj) {
         void* outs[3] = {ws + L.q, ws + L.k, ws + L.v};
         const void* Ws[3] = {Wq, nW == 3 ? Wk : Wq, nW == 3 ? Wv : Wq};

@@ -136,6 +136,195 @@ f32_attn_kernel(const float* __restrict__ Q, const float* __restrict__ K, const 
     }
 }
 
+// ---------------------------------------------------------------- one launch for small layers
+// Projections and the three phases of one (batch, head) in one CTA, everything in shared memory: the layer of a few
+// dozen vectors is a few microseconds of work, and two launches with a round trip of q, k, v through global memory
+// cost more than the arithmetic.  Element-exact skipping as in the kernels above: a weight the scheme does not need
+// is never computed, and the census counts the multiply-accumulates actually executed.
+constexpr int FS_THREADS = 256;
+constexpr int FS_MAX_FLOATS = 56 * 1024;          // shared-memory budget in floats (224 KB)
+
+struct FusedLayout {
+    int xs_ld, ds, s_ld;                          // row pitches of X, of q/k/v, of the weight matrix S
+    size_t xs, ws, qs, ks, vs, sm, rinv, total;   // offsets in floats
+};
+__host__ __device__ inline FusedLayout fused_layout(int n, int D, int d, int nW) {
+    FusedLayout L;
+    L.xs_ld = D + 1; L.ds = d + 4; L.s_ld = n + 1;
+    size_t off = 0;
+    L.xs = off; off += (size_t)n * L.xs_ld; off = (off + 3) & ~size_t(3);
+    L.ws = off; off += (size_t)nW * D * d;
+    L.qs = off; off += (size_t)n * L.ds;
+    L.ks = nW == 3 ? off : L.qs; if (nW == 3) off += (size_t)n * L.ds;
+    L.vs = nW == 3 ? off : L.qs; if (nW == 3) off += (size_t)n * L.ds;
+    L.sm = off; off += (size_t)n * L.s_ld;
+    L.rinv = off; off += n;
+    L.total = off;
+    return L;
+}
+
+__global__ void __launch_bounds__(FS_THREADS, 1)
+f32_fused_layer_kernel(const float* __restrict__ X, const float* __restrict__ Wq, const float* __restrict__ Wk,
+                       const float* __restrict__ Wv, float* __restrict__ out, int n, int H, int D, int d, float scale,
+                       int scheme, DeviceCounters* dc) {
+    extern __shared__ float4 fs_smem4[];
+    float* sm = reinterpret_cast<float*>(fs_smem4);
+    const int nW = scheme == PSA_SYMMETRIC ? 1 : 3;
+    const FusedLayout L = fused_layout(n, D, d, nW);
+    float* xs = sm + L.xs; float* ws = sm + L.ws; float* qs = sm + L.qs; float* ks = sm + L.ks; float* vs = sm + L.vs;
+    float* S = sm + L.sm; float* rinv = sm + L.rinv;
+    const int b = blockIdx.x / H, h = blockIdx.x - b * H;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool lower = scheme != PSA_FULL;            // only j <= i is computed in phase 1 (masked; symmetric: then mirrored)
+    const bool masked = scheme == PSA_MASKED;
+    const size_t HD = (size_t)H * d;
+    unsigned long long qk = 0, pv = 0, ex = 0;
+
+    // ---- stage X[b] and this head's columns of the projection matrices (loads batched eight deep: a layer this small
+    // lives on the latency of its first loads)
+    {
+        const float* xb = X + (size_t)b * n * D;
+        for (int t0 = tid; t0 < n * D; t0 += 8 * FS_THREADS) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { const int t = t0 + u * FS_THREADS; v[u] = t < n * D ? __ldg(xb + t) : 0.f; }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int t = t0 + u * FS_THREADS;
+                if (t < n * D) { const int i = t / D; xs[i * L.xs_ld + (t - i * D)] = v[u]; }
+            }
+        }
+        const int d4 = d / 4;
+        for (int w = 0; w < nW; ++w) {
+            const float* W = (w == 0 ? Wq : (w == 1 ? Wk : Wv)) + (size_t)h * d;
+            float4* dst = reinterpret_cast<float4*>(ws + (size_t)w * D * d);
+            for (int t0 = tid; t0 < D * d4; t0 += 4 * FS_THREADS) {
+                float4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int t = t0 + u * FS_THREADS;
+                    if (t < D * d4) { const int k = t / d4; v[u] = __ldg(reinterpret_cast<const float4*>(W + (size_t)k * HD) + (t - k * d4)); }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) { const int t = t0 + u * FS_THREADS; if (t < D * d4) dst[t] = v[u]; }
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- projections (Sec. 3.1): 4 x 4 register tiles of q, k, v
+    const int tr = (n + 3) / 4, tc = d / 4;
+    for (int t = tid; t < nW * tr * tc; t += FS_THREADS) {
+        const int w = t / (tr * tc), rem = t - w * tr * tc;
+        const int i0 = (rem / tc) * 4, c0 = (rem % tc) * 4;
+        const float* wp = ws + (size_t)w * D * d + c0;
+        float acc[4][4] = {};
+        int row[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) row[r] = min(i0 + r, n - 1) * L.xs_ld;
+        for (int k = 0; k < D; ++k) {
+            const float4 wv = *reinterpret_cast<const float4*>(wp + (size_t)k * d);
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const float x = xs[row[r] + k];
+                acc[r][0] = fmaf(x, wv.x, acc[r][0]); acc[r][1] = fmaf(x, wv.y, acc[r][1]);
+                acc[r][2] = fmaf(x, wv.z, acc[r][2]); acc[r][3] = fmaf(x, wv.w, acc[r][3]);
+            }
+        }
+        float* dst = w == 0 ? qs : (w == 1 ? ks : vs);
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+            if (i0 + r < n) *reinterpret_cast<float4*>(dst + (size_t)(i0 + r) * L.ds + c0) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+    }
+    __syncthreads();
+
+    // ---- phase 1 (Eq. 1): S_ij = scale q_i . k_j for the weights the scheme needs, in 4 x 4 register tiles
+    const int tn = (n + 3) / 4;
+    for (int t = tid; t < tn * tn; t += FS_THREADS) {
+        const int i0 = (t / tn) * 4, j0 = (t % tn) * 4;
+        if (lower && j0 > i0 + 3) continue;                       // wholly above the diagonal: never issued
+        // which of the tile's 16 weights exist: inside the matrix and, for the schemes that compute the lower triangle
+        // only, on or below the diagonal.  The multiply-accumulates of the others are predicated off, not executed.
+        unsigned mask = 0;
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i0 + r < n && j0 + u < n && !(lower && j0 + u > i0 + r)) mask |= 1u << (4 * r + u);
+        const int qrow[4] = {min(i0, n - 1), min(i0 + 1, n - 1), min(i0 + 2, n - 1), min(i0 + 3, n - 1)};
+        const int krow[4] = {min(j0, n - 1), min(j0 + 1, n - 1), min(j0 + 2, n - 1), min(j0 + 3, n - 1)};
+        float acc[4][4] = {};
+        for (int c = 0; c < d; ++c) {
+            float qv[4], kv[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) { qv[r] = qs[(size_t)qrow[r] * L.ds + c]; kv[r] = ks[(size_t)krow[r] * L.ds + c]; }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (mask & (1u << (4 * r + u))) acc[r][u] = fmaf(qv[r], kv[u], acc[r][u]);
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (mask & (1u << (4 * r + u))) {
+                    const float v = acc[r][u] * scale;
+                    S[(size_t)(i0 + r) * L.s_ld + j0 + u] = v;
+                    if (scheme == PSA_SYMMETRIC) S[(size_t)(j0 + u) * L.s_ld + i0 + r] = v;   // reuse (Sec. 4.1): a store, no MACs
+                }
+        qk += (unsigned long long)__popc(mask) * d;
+    }
+    __syncthreads();
+
+    // ---- phase 2 (Eq. 2): one warp per row; the division is applied to the output row
+    for (int i = warp; i < n; i += FS_THREADS / 32) {
+        const int jend = masked ? i + 1 : n;
+        float* row = S + (size_t)i * L.s_ld;
+        float mx = -INFINITY;
+        for (int j = lane; j < jend; j += 32) mx = fmaxf(mx, row[j]);
+        for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        float sum = 0.f;
+        for (int j = lane; j < jend; j += 32) {
+            const float e = expf(row[j] - mx);
+            row[j] = e;
+            sum += e;
+        }
+        for (int off = 16; off; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        if (lane == 0) { rinv[i] = 1.f / sum; ex += (unsigned long long)jend; }
+    }
+    __syncthreads();
+
+    // ---- phase 3 (Eq. 3): y_i = sum_j w_ij v_j over the kept weights, four output components per thread
+    for (int t = tid; t < n * tc; t += FS_THREADS) {
+        const int i = t / tc, c0 = (t - i * tc) * 4;
+        const int jend = masked ? i + 1 : n;
+        const float* row = S + (size_t)i * L.s_ld;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j = 0; j < jend; ++j) {
+            const float w = row[j];
+            const float4 v = *reinterpret_cast<const float4*>(vs + (size_t)j * L.ds + c0);
+            acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y); acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+        }
+        const float r = rinv[i];
+        *reinterpret_cast<float4*>(out + ((size_t)b * n + i) * HD + (size_t)h * d + c0) = make_float4(acc.x * r, acc.y * r, acc.z * r, acc.w * r);
+        pv += 4ull * jend;
+    }
+
+    // ---- census
+    for (int off = 16; off; off >>= 1) {
+        qk += __shfl_xor_sync(0xffffffffu, qk, off);
+        pv += __shfl_xor_sync(0xffffffffu, pv, off);
+        ex += __shfl_xor_sync(0xffffffffu, ex, off);
+    }
+    if (lane == 0) {
+        if (qk) atomicAdd(&dc->qk_macs, qk);
+        if (pv) atomicAdd(&dc->pv_macs, pv);
+        if (ex) atomicAdd(&dc->exps, ex);
+    }
+    if (tid == 0) atomicAdd(&dc->proj_macs, (unsigned long long)nW * n * D * d);
+}
+
 size_t attn_smem_bytes(int n, int d) {
     return sizeof(float) * ((size_t)KEY_TILE * (d + 1) + (size_t)ROWS_PER_BLOCK * d + (size_t)ROWS_PER_BLOCK * n);
 }
@@ -146,6 +335,26 @@ cudaError_t f32_project(const float* X, const float* const W[3], float* const ou
                         int N, const float* residual, DeviceCounters* dc, cudaStream_t stream) {
     dim3 block(PROJ_TILE, PROJ_TILE), grid((N + PROJ_TILE - 1) / PROJ_TILE, (rows + PROJ_TILE - 1) / PROJ_TILE, nW);
     f32_project_kernel<<<grid, block, 0, stream>>>(X, W[0], W[1], W[2], out[0], out[1], out[2], rows, D, N, residual, dc);
+    return cudaGetLastError();
+}
+
+bool f32_fused_fits(int n, int D, int d, int scheme) {
+    if (n > 256 || d % 4 != 0 || d > 128) return false;
+    return fused_layout(n, D, d, scheme == PSA_SYMMETRIC ? 1 : 3).total <= (size_t)FS_MAX_FLOATS;
+}
+
+cudaError_t f32_fused_layer(const float* X, const float* Wq, const float* Wk, const float* Wv, float* out, int B, int H,
+                            int n, int D, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream) {
+    static DeviceSetup setup;
+    if (device_setup(&setup, [] {
+            return cudaFuncSetAttribute(f32_fused_layer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        FS_MAX_FLOATS * (int)sizeof(float));
+        }, "fp32 fused layer set-up") <= 0)
+        return cudaErrorUnknown;
+    const size_t smem = fused_layout(n, D, d, scheme == PSA_SYMMETRIC ? 1 : 3).total * sizeof(float);
+    f32_fused_layer_kernel<<<B * H, FS_THREADS, smem, stream>>>(X, Wq, scheme == PSA_SYMMETRIC ? Wq : Wk,
+                                                               scheme == PSA_SYMMETRIC ? Wq : Wv, out, n, H, D, d, scale,
+                                                               scheme, dc);
     return cudaGetLastError();
 }
 

@@ -30,6 +30,12 @@ cudaError_t f32_project(const float* X, const float* const W[3], float* const ou
 cudaError_t f32_attention(const float* Q, const float* K, const float* V, float* out, float* S, int B, int H,
                           int n, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
 
+// Small layers in one launch (projections and the three phases of a (batch, head) per CTA, all in shared memory):
+// f32_fused_fits says whether a shape qualifies.  X [B, n, D], W* [D, H*d] (Wk, Wv ignored for PSA_SYMMETRIC).
+bool f32_fused_fits(int n, int D, int d, int scheme);
+cudaError_t f32_fused_layer(const float* X, const float* Wq, const float* Wk, const float* Wv, float* out, int B, int H,
+                            int n, int D, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
+
 // ---- bf16 tcgen05 path (psa_gemm.cu, psa_attn.cu) ----
 // C[w][M, N] = A[M, K] * Bw[w][K, N] (+ residual[M, N], bf16, may be null), bf16 row-major, fp32 accumulation.
 // Returns a psa_status.
