@@ -141,22 +141,24 @@ f32_attn_kernel(const float* __restrict__ Q, const float* __restrict__ K, const 
 // dozen vectors is a few microseconds of work, and two launches with a round trip of q, k, v through global memory
 // cost more than the arithmetic.  Element-exact skipping as in the kernels above: a weight the scheme does not need
 // is never computed, and the census counts the multiply-accumulates actually executed.
-constexpr int FS_THREADS = 256;
+constexpr int FS_THREADS = 512;
 constexpr int FS_MAX_FLOATS = 56 * 1024;          // shared-memory budget in floats (224 KB)
 
 struct FusedLayout {
-    int xs_ld, ds, s_ld;                          // row pitches of X, of q/k/v, of the weight matrix S
-    size_t xs, ws, qs, ks, vs, sm, rinv, total;   // offsets in floats
+    int xs_ld, t_ld, ds, s_ld;                    // row pitches: X, transposed q and k, v, the weight matrix S
+    size_t xs, ws, qt, kt, vs, sm, rinv, total;   // offsets in floats
 };
+// q and k are kept transposed ([component][vector]) so that phase 1 reads four consecutive vectors of one component
+// as one 16-byte access; v is kept [vector][component] for phase 3.
 __host__ __device__ inline FusedLayout fused_layout(int n, int D, int d, int nW) {
     FusedLayout L;
-    L.xs_ld = D + 1; L.ds = d + 4; L.s_ld = n + 1;
+    L.xs_ld = D + 1; L.t_ld = ((n + 3) & ~3) + 4; L.ds = d + 4; L.s_ld = n + 1;
     size_t off = 0;
     L.xs = off; off += (size_t)n * L.xs_ld; off = (off + 3) & ~size_t(3);
     L.ws = off; off += (size_t)nW * D * d;
-    L.qs = off; off += (size_t)n * L.ds;
-    L.ks = nW == 3 ? off : L.qs; if (nW == 3) off += (size_t)n * L.ds;
-    L.vs = nW == 3 ? off : L.qs; if (nW == 3) off += (size_t)n * L.ds;
+    L.qt = off; off += (size_t)d * L.t_ld;
+    L.kt = nW == 3 ? off : L.qt; if (nW == 3) off += (size_t)d * L.t_ld;
+    L.vs = off; off += (size_t)n * L.ds;
     L.sm = off; off += (size_t)n * L.s_ld;
     L.rinv = off; off += n;
     L.total = off;
@@ -171,7 +173,7 @@ f32_fused_layer_kernel(const float* __restrict__ X, const float* __restrict__ Wq
     float* sm = reinterpret_cast<float*>(fs_smem4);
     const int nW = scheme == PSA_SYMMETRIC ? 1 : 3;
     const FusedLayout L = fused_layout(n, D, d, nW);
-    float* xs = sm + L.xs; float* ws = sm + L.ws; float* qs = sm + L.qs; float* ks = sm + L.ks; float* vs = sm + L.vs;
+    float* xs = sm + L.xs; float* ws = sm + L.ws; float* qt = sm + L.qt; float* kt = sm + L.kt; float* vs = sm + L.vs;
     float* S = sm + L.sm; float* rinv = sm + L.rinv;
     const int b = blockIdx.x / H, h = blockIdx.x - b * H;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -231,10 +233,17 @@ f32_fused_layer_kernel(const float* __restrict__ X, const float* __restrict__ Wq
                 acc[r][2] = fmaf(x, wv.z, acc[r][2]); acc[r][3] = fmaf(x, wv.w, acc[r][3]);
             }
         }
-        float* dst = w == 0 ? qs : (w == 1 ? ks : vs);
+        if (w < 2) {          // q, k: transposed (rows beyond n land in the pitch's padding and are never used)
+            float* dst = w == 0 ? qt : kt;
 #pragma unroll
-        for (int r = 0; r < 4; ++r)
-            if (i0 + r < n) *reinterpret_cast<float4*>(dst + (size_t)(i0 + r) * L.ds + c0) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+            for (int u = 0; u < 4; ++u)
+                *reinterpret_cast<float4*>(dst + (size_t)(c0 + u) * L.t_ld + i0) = make_float4(acc[0][u], acc[1][u], acc[2][u], acc[3][u]);
+        }
+        if (w == 2 || nW == 1) {   // v (the symmetric scheme's single projection is q, k and v at once)
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                if (i0 + r < n) *reinterpret_cast<float4*>(vs + (size_t)(i0 + r) * L.ds + c0) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+        }
     }
     __syncthreads();
 
@@ -243,37 +252,63 @@ f32_fused_layer_kernel(const float* __restrict__ X, const float* __restrict__ Wq
     for (int t = tid; t < tn * tn; t += FS_THREADS) {
         const int i0 = (t / tn) * 4, j0 = (t % tn) * 4;
         if (lower && j0 > i0 + 3) continue;                       // wholly above the diagonal: never issued
-        // which of the tile's 16 weights exist: inside the matrix and, for the schemes that compute the lower triangle
-        // only, on or below the diagonal.  The multiply-accumulates of the others are predicated off, not executed.
-        unsigned mask = 0;
+        const bool inside = i0 + 3 < n && j0 + 3 < n;
+        if (inside && !(lower && j0 == i0)) {
+            // a whole tile: 16 weights
+            float acc[4][4] = {};
+            for (int c = 0; c < d; ++c) {
+                const float4 q4 = *reinterpret_cast<const float4*>(qt + (size_t)c * L.t_ld + i0);
+                const float4 k4 = *reinterpret_cast<const float4*>(kt + (size_t)c * L.t_ld + j0);
+                const float qv[4] = {q4.x, q4.y, q4.z, q4.w}, kv[4] = {k4.x, k4.y, k4.z, k4.w};
 #pragma unroll
-        for (int r = 0; r < 4; ++r)
+                for (int r = 0; r < 4; ++r)
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (i0 + r < n && j0 + u < n && !(lower && j0 + u > i0 + r)) mask |= 1u << (4 * r + u);
-        const int qrow[4] = {min(i0, n - 1), min(i0 + 1, n - 1), min(i0 + 2, n - 1), min(i0 + 3, n - 1)};
-        const int krow[4] = {min(j0, n - 1), min(j0 + 1, n - 1), min(j0 + 2, n - 1), min(j0 + 3, n - 1)};
-        float acc[4][4] = {};
-        for (int c = 0; c < d; ++c) {
-            float qv[4], kv[4];
-#pragma unroll
-            for (int r = 0; r < 4; ++r) { qv[r] = qs[(size_t)qrow[r] * L.ds + c]; kv[r] = ks[(size_t)krow[r] * L.ds + c]; }
+                    for (int u = 0; u < 4; ++u) acc[r][u] = fmaf(qv[r], kv[u], acc[r][u]);
+            }
 #pragma unroll
             for (int r = 0; r < 4; ++r)
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (mask & (1u << (4 * r + u))) acc[r][u] = fmaf(qv[r], kv[u], acc[r][u]);
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (mask & (1u << (4 * r + u))) {
+                for (int u = 0; u < 4; ++u) {
                     const float v = acc[r][u] * scale;
                     S[(size_t)(i0 + r) * L.s_ld + j0 + u] = v;
                     if (scheme == PSA_SYMMETRIC) S[(size_t)(j0 + u) * L.s_ld + i0 + r] = v;   // reuse (Sec. 4.1): a store, no MACs
                 }
-        qk += (unsigned long long)__popc(mask) * d;
+            qk += 16ull * d;
+        } else if (inside) {
+            // the tile on the diagonal of a lower-triangle scheme: the 10 weights with j <= i, nothing above them
+            float acc[4][4] = {};
+            for (int c = 0; c < d; ++c) {
+                const float4 q4 = *reinterpret_cast<const float4*>(qt + (size_t)c * L.t_ld + i0);
+                const float4 k4 = *reinterpret_cast<const float4*>(kt + (size_t)c * L.t_ld + j0);
+                const float qv[4] = {q4.x, q4.y, q4.z, q4.w}, kv[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+#pragma unroll
+                    for (int u = 0; u <= r; ++u) acc[r][u] = fmaf(qv[r], kv[u], acc[r][u]);
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int u = 0; u <= r; ++u) {
+                    const float v = acc[r][u] * scale;
+                    S[(size_t)(i0 + r) * L.s_ld + j0 + u] = v;
+                    if (scheme == PSA_SYMMETRIC) S[(size_t)(j0 + u) * L.s_ld + i0 + r] = v;
+                }
+            qk += 10ull * d;
+        } else {
+            // a tile that the edge of the matrix crosses (n not a multiple of 4): weight by weight
+            for (int r = 0; r < 4; ++r)
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + r, j = j0 + u;
+                    if (i >= n || j >= n || (lower && j > i)) continue;
+                    float acc = 0.f;
+                    for (int c = 0; c < d; ++c) acc = fmaf(qt[(size_t)c * L.t_ld + i], kt[(size_t)c * L.t_ld + j], acc);
+                    acc *= scale;
+                    S[(size_t)i * L.s_ld + j] = acc;
+                    if (scheme == PSA_SYMMETRIC) S[(size_t)j * L.s_ld + i] = acc;
+                    qk += d;
+                }
+        }
     }
     __syncthreads();
 
