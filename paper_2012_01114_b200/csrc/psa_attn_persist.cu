@@ -47,12 +47,9 @@ struct PCfg {
     static constexpr int TILE_BYTES = 128 * D * 2;      // one Q, K or V tile
     static constexpr int KSTAGES = D == 128 ? 2 : 4;
     static constexpr int VSTAGES = D == 128 ? 2 : 4;
-    // output staging buffers.  d = 64: a unit is the two warps that share 32 rows (32 rows x 64 columns), one buffer
-    // for each of an item's 8 units.  d = 128: a unit is one warp (its 32 rows x 64 columns), and the 16 units of an
-    // item take 6 buffers in turn (shared memory has no room for more)
-    static constexpr bool WARP_UNITS = D == 128;
-    static constexpr int STAGE_BYTES = 32 * 64 * 2;
-    static constexpr int STAGE_BUFS = D == 64 ? 8 : 6;
+    // output staging: one [16 rows x 64 columns] bf16 buffer per softmax warp, used for each 64-column half in turn
+    static constexpr int STAGE_BYTES = 16 * 64 * 2;
+    static constexpr int STAGE_BUFS = 2 * SOFTMAX_WARPS_PER_TILE;
     static constexpr int SMEM = (2 + KSTAGES + VSTAGES) * TILE_BYTES + STAGE_BUFS * STAGE_BYTES + 1024;
     static constexpr bool SEP_P = D == 64;
     static constexpr int TMEM_S = 0, TMEM_P = 256, TMEM_O = SEP_P ? 384 : 256;
@@ -68,21 +65,6 @@ struct PBars {
     uint64_t k_full[8], k_empty[8], v_full[4], v_empty[4];
     uint64_t s_full[2], s_free[2], p_ready[2], o_done[2];
 };
-
-// Bounded wait until a shared-memory counter, which only grows, has reached `target`.
-__device__ __forceinline__ bool count_wait(const volatile uint32_t* counter, uint32_t target, volatile int* abort_flag) {
-    if (*counter >= target) return true;
-    const uint64_t t0 = globaltimer_ns();
-    uint32_t it = 0;
-    while (*counter < target) {
-        __nanosleep(20);
-        if ((++it & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > PSA_WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
-        }
-    }
-    return true;
-}
 
 // d = 64 has an MMA-issuing thread per row tile slot (warp 1 for slot 0, the last warp for slot 1): a block there is
 // half the tensor work of d = 128 but as many instructions to issue, and one thread was measured to be the limit.
@@ -111,9 +93,6 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
     __shared__ int item_ring[2];
-    __shared__ volatile uint32_t stage_released[8];   // per staging buffer: uses whose store has read it
-    __shared__ float xch_max[2][2][2][128];   // [block parity][tile][column half][row]
-    __shared__ float xch_sum[2][2][128];      // [tile][column half][row]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n = sp.n, T = sp.T;
@@ -126,7 +105,6 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
         abort_flag = 0;
         // the counter block of the NEXT call on this workspace is cleared here, off that call's critical path
         if (blockIdx.x == 0 && dc_next) *dc_next = DeviceCounters{0, 0, 0, 0, 0, 0, 0};
-        for (int i = 0; i < 8; ++i) stage_released[i] = 0;
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bars.item_full[t], 1);
             mbar_init(&bars.item_empty[t], item_readers<D>());
@@ -359,12 +337,12 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                 if (first) {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
-                        umma_ts(dO, aP + (SEP ? kk * 8 : (kk >> 2) * 64 + (kk & 3) * 8),
+                        umma_ts(dO, aP + kk * 8,
                                 umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, kk != 0);
                 } else {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
-                        umma_ts(dO, aP + (SEP ? kk * 8 : (kk >> 2) * 64 + (kk & 3) * 8),
+                        umma_ts(dO, aP + kk * 8,
                                 umma_desc_join(v + kk * (2048 >> 4), UMMA_DESC_HI_SW128), idescO, 1);
                 }
                 ++pv_blocks;
@@ -430,48 +408,39 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
         }
     } else {
         // ------------------------------------------------------------ softmax + epilogue
-        // TPR threads share a query row; thread `part` owns block columns [part*CPT, (part+1)*CPT).
-        constexpr int CPT = 128 / TPR;                           // score columns per thread
-        constexpr int NCH = CPT / 32;                            // 32-column chunks per thread
-        constexpr int OPT = D / TPR;                             // output columns per thread
+        // Eight warps per row tile.  A warp owns 16 rows (TMEM lanes) and reads them in the quad layout (sm100.cuh): the
+        // four threads of a quad share two rows, A and B = A + 8, each holding every fourth pair of their columns, so a
+        // row maximum or row sum is two shuffles inside the quad and the warps never wait for one another.
         const int sw = warp - CTRL_WARPS;
         const int t = sw / SOFTMAX_WARPS_PER_TILE;              // row tile slot of this warp
-        const int part = (sw % SOFTMAX_WARPS_PER_TILE) >> 2;    // which share of the row's columns
+        const int wq = sw % SOFTMAX_WARPS_PER_TILE;             // warp inside the slot
         const int q = warp & 3;                                 // TMEM lane quarter this warp may access
-        const int r = q * 32 + lane;                            // row inside the tile = TMEM lane
-        const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
+        const int row0 = q * 32 + (wq >> 2) * 16;               // first of the warp's 16 rows inside the tile
+        const int rA = row0 + (lane >> 2), rB = rA + 8;         // this thread's rows
+        const int cq = 2 * (lane & 3);                          // its first column inside every group of 8
+        const uint32_t lane_off = static_cast<uint32_t>(row0) << 16;
         const uint32_t tS = tmem + Cfg::TMEM_S + t * 128 + lane_off;
-        const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off + part * OPT;
-        const uint32_t tP = tmem + Cfg::TMEM_P + t * 64 + lane_off;     // separate-P layout only
-        const int pair_bar = 1 + t * 4 + q;                     // named barrier of the warps sharing rows
-        const int col_base = part * CPT;
+        const uint32_t tO = tmem + Cfg::TMEM_O + t * D + lane_off;
+        const uint32_t tP = SEP ? tmem + Cfg::TMEM_P + t * 64 + lane_off : tS;     // P: 64 columns, over S at d = 128
+        uint8_t* stage = sStage + (t * SOFTMAX_WARPS_PER_TILE + wq) * Cfg::STAGE_BYTES;   // this warp's output staging buffer
         uint32_t my_items = 0;                                  // items this tile slot took part in
         uint32_t blk = 0;                                       // blocks this tile slot has processed, all items
+        bool store_pending = false;                             // a TMA store of this warp may still be reading `stage`
         bool ok = true;
-        for (uint32_t it = 0;; ++it) {
-            if (ok) ok = mbar_wait(&bars.item_full[it & 1], (it >> 1) & 1, abortp);
-            // the two warps that share rows take the item or neither does (one may have given up a wait); pairs of
-            // a slot are not held together here: a pair whose output is on its way starts on the next item
-            ok = named_bar_all(ok, pair_bar, 32 * TPR);
+        for (uint32_t it = 0; ok; ++it) {
+            ok = mbar_wait(&bars.item_full[it & 1], (it >> 1) & 1, abortp);
+            ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const int idx = item_ring[it & 1];
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars.item_empty[it & 1]);
             if (idx < 0) break;
             const CtaWork work = item_work(idx);
-            if (t >= work.ntiles) {
-                // no rows for this slot in this item: its units' turns at the staging buffers are passed on
-                if ((Cfg::WARP_UNITS || part == 0) && lane == 0) {
-                    const uint32_t unit = Cfg::WARP_UNITS ? it * 16u + 8u * t + 4u * part + q : it * 8u + 4u * t + q;
-                    const uint32_t sbuf = unit % Cfg::STAGE_BUFS, suse = unit / Cfg::STAGE_BUFS;
-                    if (count_wait(&stage_released[sbuf], suse, abortp)) stage_released[sbuf] = suse + 1;
-                }
-                continue;
-            }
+            if (t >= work.ntiles) continue;                     // no rows for this slot in this item
             const int b = work.bh / H, h = work.bh - b * H;
             const int It = work.tile0 + t;
             const int nkv = kv_tiles(It, T, scheme);
-            float m_run = -INFINITY, l_run = 0.f;
+            float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;       // running maxima (log2 units) and row sums
             for (int j = 0; j < nkv; ++j, ++blk) {
                 if (SEP) {
                     ok = mbar_wait(&bars.s_full[t], blk & 1, abortp);                 // every S has its own commit
@@ -481,138 +450,124 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                     else ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
                 }
                 ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
                 // Element predicate: on the diagonal block of the masked scheme keys beyond the row's own index,
-                // and on a ragged last block keys beyond the sequence, carry no weight.  `cb` = last kept column.
+                // and on a ragged last block keys beyond the sequence, carry no weight.  cbA, cbB = last kept columns.
                 const int nvalid = min(TILE, n - j * TILE);
                 const bool on_diag = masked && (j == It);
                 const bool diag = on_diag || nvalid < TILE;
-                const int cb = min(on_diag ? r : TILE - 1, nvalid - 1);
-                float mx = -INFINITY;
-                uint32_t sreg[NCH][32];
-                if (ok) {
-                    // ---- pass 1: maximum of this thread's scores
-                    tc_fence_after();
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) tmem_ld32(tS + col_base + 32 * c, sreg[c]);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c)
-                        mx = diag ? max_chunk32<true>(sreg[c], col_base + 32 * c, cb, mx)
-                                  : max_chunk32<false>(sreg[c], col_base + 32 * c, r, mx);
-                }
-                // The two threads of a row meet here to exchange their half-row maxima (and to leave
-                // together if either gave up a wait).
-                xch_max[blk & 1][t][part][r] = mx;
-                ok = named_bar_all(ok, pair_bar, 64);
-                if (!ok) break;
-                mx = fmaxf(mx, xch_max[blk & 1][t][part ^ 1][r]);
-                const float mx2 = mx * sl2;
-                float alpha = 1.f;
-                if (mx2 > m_run + RESCALE_THRESHOLD) {   // also taken on the first block (m_run = -inf)
-                    alpha = ex2_mufu(m_run - mx2);
-                    m_run = mx2;
-                }
-                // ---- pass 2: P = exp2(S*sl2 - m) as bf16
-                float rowsum = 0.f;
-                // the scores were only reduced so far: fetch them again
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) tmem_ld32(tS + col_base + 32 * c, sreg[c]);
+                const int cbA = min(on_diag ? rA : TILE - 1, nvalid - 1);
+                const int cbB = min(on_diag ? rB : TILE - 1, nvalid - 1);
+                // ---- the rows' 2 x 64 scores of this block
+                uint32_t s0[32], s1[32];
+                tc_fence_after();
+                tmem_ld_quad64(tS, s0);
+                tmem_ld_quad64(tS + 64, s1);
                 tc_wait_ld();
                 if (SEP) {
                     // S is in registers: the issuer may overwrite it with the next scores while the exponentials run
                     tc_fence_before();
                     mbar_arrive(&bars.s_free[t]);
-                    // P and O are still in use by PV_{j-1} until its commit.  A wait given up here is not
-                    // acted on before the next pair barrier, so that the two threads of a row stay together.
-                    if (j > 0) {
-                        ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
-                        ok = __all_sync(0xffffffffu, ok);
-                        tc_fence_after();
-                    }
                 }
-                if (ok) {
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        uint32_t pk[16];
-                        const int kc = col_base + 32 * c;            // first key column of the chunk
-                        rowsum += diag ? exp_chunk32<true>(sreg[c], sl2, -m_run, kc, cb, pk)
-                                       : exp_chunk32<false>(sreg[c], sl2, -m_run, kc, r, pk);
-                        // P over S: keys [kc, kc+32) go to S columns (kc/64)*64 + (kc%64)/2, behind this thread's own reads
-                        tmem_st16(SEP ? tP + (kc >> 1) : tS + (kc >> 6) * 64 + ((kc & 63) >> 1), pk);
-                    }
+                // ---- pass 1: row maxima of the block, completed inside the quad
+                float bA = -INFINITY, bB = -INFINITY;
+                if (diag) {
+                    max_quad64<true>(s0, cq, cbA, cbB, bA, bB);
+                    max_quad64<true>(s1, 64 + cq, cbA, cbB, bA, bB);
+                } else {
+                    max_quad64<false>(s0, cq, cbA, cbB, bA, bB);
+                    max_quad64<false>(s1, 64 + cq, cbA, cbB, bA, bB);
                 }
-                l_run = fmaf(l_run, alpha, rowsum);
-                if (ok && j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // rare: a row maximum grew by > 2^8
-                    const unsigned grown = __ballot_sync(0xffffffffu, alpha != 1.f);
-                    if (part == 0 && lane == 0) atomicAdd(&dc->rescales, (unsigned long long)__popc(grown));
-#pragma unroll
-                    for (int c = 0; c < OPT / 32; ++c) {
+                bA = quad_max(bA) * sl2;
+                bB = quad_max(bB) * sl2;
+                float alphaA = 1.f, alphaB = 1.f;
+                if (bA > mA + RESCALE_THRESHOLD) {   // also taken on the first block (m = -inf)
+                    alphaA = ex2_mufu(mA - bA);
+                    mA = bA;
+                }
+                if (bB > mB + RESCALE_THRESHOLD) {
+                    alphaB = ex2_mufu(mB - bB);
+                    mB = bB;
+                }
+                // ---- pass 2: P = exp2(S*sl2 - m) as bf16, keys 0-63 then keys 64-127
+                float sumA = 0.f, sumB = 0.f;
+                uint32_t pk[16];
+                if (diag) exp_quad64<true>(s0, sl2, -mA, -mB, cq, cbA, cbB, pk, sumA, sumB);
+                else exp_quad64<false>(s0, sl2, -mA, -mB, cq, cbA, cbB, pk, sumA, sumB);
+                if (SEP && blk > 0) {
+                    // P and O are still in use by the PV before this one until its commit
+                    ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                tmem_st_quad32(tP, pk);
+                if (diag) exp_quad64<true>(s1, sl2, -mA, -mB, 64 + cq, cbA, cbB, pk, sumA, sumB);
+                else exp_quad64<false>(s1, sl2, -mA, -mB, 64 + cq, cbA, cbB, pk, sumA, sumB);
+                tmem_st_quad32(tP + 32, pk);
+                lA = fmaf(lA, alphaA, sumA);
+                lB = fmaf(lB, alphaB, sumB);
+                if (j > 0 && __any_sync(0xffffffffu, alphaA != 1.f || alphaB != 1.f)) {   // rare: a row maximum grew by > 2^8
+                    const int nA = __popc(__ballot_sync(0xffffffffu, (lane & 3) == 0 && alphaA != 1.f));
+                    const int nB = __popc(__ballot_sync(0xffffffffu, (lane & 3) == 0 && alphaB != 1.f));
+                    if (lane == 0) atomicAdd(&dc->rescales, (unsigned long long)(nA + nB));
+#pragma unroll 1
+                    for (int c = 0; c < D / 64; ++c) {
                         uint32_t v[32];
-                        tmem_ld32(tO + 32 * c, v);
+                        tmem_ld_quad64(tO + 64 * c, v);
                         tc_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                        tmem_st32(tO + 32 * c, v);
+                        for (int g = 0; g < 8; ++g) {
+                            v[4 * g] = __float_as_uint(__uint_as_float(v[4 * g]) * alphaA);
+                            v[4 * g + 1] = __float_as_uint(__uint_as_float(v[4 * g + 1]) * alphaA);
+                            v[4 * g + 2] = __float_as_uint(__uint_as_float(v[4 * g + 2]) * alphaB);
+                            v[4 * g + 3] = __float_as_uint(__uint_as_float(v[4 * g + 3]) * alphaB);
+                        }
+                        tmem_st_quad64(tO + 64 * c, v);
                     }
                 }
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(&bars.p_ready[t]);
             }
-            if (ok) ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
-            xch_sum[t][part][r] = l_run;
-            ok = named_bar_all(ok, pair_bar, 32 * TPR);
             if (!ok) break;
-            // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row), bf16.  A unit (a warp, or
-            // the two warps that share 32 rows) writes its rows into a staging buffer and one lane hands it to
-            // TMA.  Buffers are taken in the fixed order of the units; a unit waits until the store of the unit
-            // that last used its buffer has read it.
+            ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            // ---- epilogue: y = O / l (the division of Eq. 2, applied once per output row), bf16.  The warp writes its
+            // 16 rows, 64 columns at a time, into its own staging buffer and one lane hands the buffer to TMA.
             tc_fence_after();
-            const float inv = 1.f / (l_run + xch_sum[t][part ^ 1][r]);
-            const uint32_t unit = Cfg::WARP_UNITS ? it * 16u + 8u * t + 4u * part + q : it * 8u + 4u * t + q;
-            const uint32_t sbuf = unit % Cfg::STAGE_BUFS, suse = unit / Cfg::STAGE_BUFS;
-            uint8_t* stage = sStage + sbuf * Cfg::STAGE_BYTES;
-            ok = count_wait(&stage_released[sbuf], suse, abortp);
-            if (ok) {
+            const float invA = 1.f / quad_sum(lA), invB = 1.f / quad_sum(lB);
 #pragma unroll
-                for (int c = 0; c < OPT / 32; ++c) {
-                    const int col = part * OPT + 32 * c;            // first of 32 output columns handled here
-                    uint32_t v[32];
-                    tmem_ld32(tO + 32 * c, v);
-                    tc_wait_ld();
-                    uint8_t* sub = stage + (Cfg::WARP_UNITS ? 0 : (col / 64) * 4096);   // [32 rows x 64 columns] sub-tiles, 128-byte swizzle
+            for (int u = 0; u < Cfg::SUB; ++u) {
+                uint32_t v[32];
+                tmem_ld_quad64(tO + 64 * u, v);
+                tc_wait_ld();
+                if (store_pending) {        // the store that last used the buffer must have read it
+                    if (lane == 0) tma_store_wait_read();
+                    __syncwarp();
+                }
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint4 o;
-                        o.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]) * inv, __uint_as_float(v[g * 8 + 1]) * inv);
-                        o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]) * inv, __uint_as_float(v[g * 8 + 3]) * inv);
-                        o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]) * inv, __uint_as_float(v[g * 8 + 5]) * inv);
-                        o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]) * inv, __uint_as_float(v[g * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(sub + swz128_offset(lane, (col % 64) / 8 + g)) = o;
-                    }
+                for (int g = 0; g < 8; ++g) {       // columns 8g + cq, 8g + cq + 1 of rows A and B: 16-byte chunk g of the row
+                    const uint32_t a = pack_bf16x2(__uint_as_float(v[4 * g]) * invA, __uint_as_float(v[4 * g + 1]) * invA);
+                    const uint32_t bb = pack_bf16x2(__uint_as_float(v[4 * g + 2]) * invB, __uint_as_float(v[4 * g + 3]) * invB);
+                    *reinterpret_cast<uint32_t*>(stage + swz128_offset(lane >> 2, g) + 2 * cq) = a;
+                    *reinterpret_cast<uint32_t*>(stage + swz128_offset((lane >> 2) + 8, g) + 2 * cq) = bb;
                 }
                 fence_async_smem();
-            }
-            // (a warp or pair that gave up carries that into the vote at the top of the next item)
-            if (Cfg::WARP_UNITS) ok = __all_sync(0xffffffffu, ok);
-            else ok = named_bar_all(ok, pair_bar, 32 * TPR);
-            if (ok && (Cfg::WARP_UNITS || part == 0) && lane == 0) {
-                if (Cfg::WARP_UNITS) {
-                    tma_store_4d(&maps.o, stage, part * OPT, h, It * TILE + q * 32, b);
-                } else {
-                    for (int u = 0; u < Cfg::SUB; ++u)
-                        tma_store_4d(&maps.o, stage + u * 4096, 64 * u, h, It * TILE + q * 32, b);
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_4d(&maps.o, stage, 64 * u, h, It * TILE + row0, b);
+                    tma_store_commit();
                 }
-                tma_store_commit();
-                tma_store_wait_read();   // the buffer may be rewritten; the global writes complete on their own
-                __threadfence_block();
-                stage_released[sbuf] = suse + 1;
+                store_pending = true;
             }
             // (the next write to O_t, PV_0 of the tile's next item, waits for P of that item, which every
             // thread of the tile signals only after these reads)
             tc_fence_before();
             ++my_items;
         }
+        if (store_pending && lane == 0) tma_store_wait_read();   // shared memory may be released; the writes complete on their own
     }
     tc_fence_before();
     __syncthreads();
@@ -633,7 +588,7 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
     if (sm_count <= 0) return PSA_ERR_CUDA;
     PMaps maps;
     if (!make_tensor_map_bf16_4d(&maps.q, Q, B, n, H, d, 128) || !make_tensor_map_bf16_4d(&maps.k, K, B, n, H, d, 128) ||
-        !make_tensor_map_bf16_4d(&maps.v, V, B, n, H, d, 128) || !make_tensor_map_bf16_4d(&maps.o, out, B, n, H, d, 32))
+        !make_tensor_map_bf16_4d(&maps.v, V, B, n, H, d, 128) || !make_tensor_map_bf16_4d(&maps.o, out, B, n, H, d, 16))
         return PSA_ERR_CUDA;
     const long long pairs = (long long)B * H * ctas_per_head(n);
     const long long split = D == 64 ? split_point(scheme, pairs, n, sm_count) : pairs;
