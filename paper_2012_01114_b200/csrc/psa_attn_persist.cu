@@ -472,12 +472,11 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                 // ---- pass 1: row maxima of the block, completed inside the quad
                 float bA = -INFINITY, bB = -INFINITY;
                 if (diag) {
-                    max_quad64<true>(s0, cq, cbA, cbB, bA, bB);
-                    max_quad64<true>(s1, 64 + cq, cbA, cbB, bA, bB);
-                } else {
-                    max_quad64<false>(s0, cq, cbA, cbB, bA, bB);
-                    max_quad64<false>(s1, 64 + cq, cbA, cbB, bA, bB);
+                    mask_quad64(s0, cq, cbA, cbB);
+                    mask_quad64(s1, 64 + cq, cbA, cbB);
                 }
+                max_quad64(s0, bA, bB);
+                max_quad64(s1, bA, bB);
                 bA = quad_max(bA) * sl2;
                 bB = quad_max(bB) * sl2;
                 float alphaA = 1.f, alphaB = 1.f;
@@ -492,8 +491,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                 // ---- pass 2: P = exp2(S*sl2 - m) as bf16, keys 0-63 then keys 64-127
                 float sumA = 0.f, sumB = 0.f;
                 uint32_t pk[16];
-                if (diag) exp_quad64<true>(s0, sl2, -mA, -mB, cq, cbA, cbB, pk, sumA, sumB);
-                else exp_quad64<false>(s0, sl2, -mA, -mB, cq, cbA, cbB, pk, sumA, sumB);
+                exp_quad64(s0, sl2, -mA, -mB, pk, sumA, sumB);
                 if (SEP && blk > 0) {
                     // P and O are still in use by the PV before this one until its commit
                     ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
@@ -502,8 +500,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                     tc_fence_after();
                 }
                 tmem_st_quad32(tP, pk);
-                if (diag) exp_quad64<true>(s1, sl2, -mA, -mB, 64 + cq, cbA, cbB, pk, sumA, sumB);
-                else exp_quad64<false>(s1, sl2, -mA, -mB, 64 + cq, cbA, cbB, pk, sumA, sumB);
+                exp_quad64(s1, sl2, -mA, -mB, pk, sumA, sumB);
                 tmem_st_quad32(tP + 32, pk);
                 lA = fmaf(lA, alphaA, sumA);
                 lB = fmaf(lB, alphaB, sumB);

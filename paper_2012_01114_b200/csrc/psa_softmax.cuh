@@ -68,54 +68,45 @@ __device__ __forceinline__ float max_chunk32(const uint32_t (&s)[32], int col0, 
     return fmaxf(max3(a[0], a[1], a[2]), a[3]);
 }
 
-// ---- the same two passes for the quad layout of tmem_ld_quad64: a thread holds 16 scores of row A (s[4g], s[4g+1])
-// and 16 of row B = A + 8 (s[4g+2], s[4g+3]), columns col0 + 8g + 2(lane%4) + {0, 1}.  With DIAG, columns beyond cbA / cbB
-// (the rows' last kept columns) carry no weight.
-template <bool DIAG>
-__device__ __forceinline__ void max_quad64(const uint32_t (&s)[32], int col0q, int cbA, int cbB, float& mA, float& mB) {
+// Softmax over a block of S held in the quad layout (sm100.cuh): s[0..31] are 16 scores of row A (s[4g], s[4g+1])
+// and 16 of row B = A + 8 (s[4g+2], s[4g+3]), columns col0 + 8g + 2(lane%4) + {0, 1}.
+//
+// Columns beyond cbA / cbB (the rows' last kept columns on a diagonal or ragged block) carry no weight: they are set
+// to -inf once, which the maximum ignores and the exponential turns into 0, so that such blocks share all other code.
+__device__ __forceinline__ void mask_quad64(uint32_t (&s)[32], int col0q, int cbA, int cbB) {
+    const uint32_t ninf = 0xff800000u;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        const int c = col0q + 8 * g;
+        if (c > cbA) s[4 * g] = ninf;
+        if (c + 1 > cbA) s[4 * g + 1] = ninf;
+        if (c > cbB) s[4 * g + 2] = ninf;
+        if (c + 1 > cbB) s[4 * g + 3] = ninf;
+    }
+}
+__device__ __forceinline__ void max_quad64(const uint32_t (&s)[32], float& mA, float& mB) {
     float a0 = mA, a1 = -INFINITY, b0 = mB, b1 = -INFINITY;
 #pragma unroll
     for (int g = 0; g < 8; g += 2) {
-        float x0 = __uint_as_float(s[4 * g]), x1 = __uint_as_float(s[4 * g + 1]);
-        float y0 = __uint_as_float(s[4 * g + 2]), y1 = __uint_as_float(s[4 * g + 3]);
-        float x2 = __uint_as_float(s[4 * g + 4]), x3 = __uint_as_float(s[4 * g + 5]);
-        float y2 = __uint_as_float(s[4 * g + 6]), y3 = __uint_as_float(s[4 * g + 7]);
-        if (DIAG) {
-            const int c = col0q + 8 * g;
-            if (c > cbA) x0 = -INFINITY;
-            if (c + 1 > cbA) x1 = -INFINITY;
-            if (c + 8 > cbA) x2 = -INFINITY;
-            if (c + 9 > cbA) x3 = -INFINITY;
-            if (c > cbB) y0 = -INFINITY;
-            if (c + 1 > cbB) y1 = -INFINITY;
-            if (c + 8 > cbB) y2 = -INFINITY;
-            if (c + 9 > cbB) y3 = -INFINITY;
-        }
-        a0 = max3(a0, x0, x1); a1 = max3(a1, x2, x3);
-        b0 = max3(b0, y0, y1); b1 = max3(b1, y2, y3);
+        a0 = max3(a0, __uint_as_float(s[4 * g]), __uint_as_float(s[4 * g + 1]));
+        b0 = max3(b0, __uint_as_float(s[4 * g + 2]), __uint_as_float(s[4 * g + 3]));
+        a1 = max3(a1, __uint_as_float(s[4 * g + 4]), __uint_as_float(s[4 * g + 5]));
+        b1 = max3(b1, __uint_as_float(s[4 * g + 6]), __uint_as_float(s[4 * g + 7]));
     }
     mA = fmaxf(a0, a1);
     mB = fmaxf(b0, b1);
 }
 // P = exp2(s*sl2 - m) for the 32 scores, packed to bf16 pairs in the layout tmem_st_quad32 expects (pk[2g] row A,
 // pk[2g+1] row B); the rows' sums of weights (before rounding) are added to sumA / sumB.
-template <bool DIAG>
-__device__ __forceinline__ void exp_quad64(const uint32_t (&s)[32], float sl2, float negmA, float negmB, int col0q, int cbA,
-                                           int cbB, uint32_t (&pk)[16], float& sumA, float& sumB) {
+__device__ __forceinline__ void exp_quad64(const uint32_t (&s)[32], float sl2, float negmA, float negmB, uint32_t (&pk)[16],
+                                           float& sumA, float& sumB) {
     float sa0 = 0.f, sa1 = 0.f, sb0 = 0.f, sb1 = 0.f;
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
-        float p0 = ex2_mufu(fmaf(__uint_as_float(s[4 * g]), sl2, negmA));
-        float p1 = ex2_mufu(fmaf(__uint_as_float(s[4 * g + 1]), sl2, negmA));
-        float p2 = ex2_mufu(fmaf(__uint_as_float(s[4 * g + 2]), sl2, negmB));
-        float p3 = ex2_mufu(fmaf(__uint_as_float(s[4 * g + 3]), sl2, negmB));
-        if (DIAG) {
-            const int c = col0q + 8 * g;
-            if (c > cbA) p0 = 0.f;
-            if (c + 1 > cbA) p1 = 0.f;
-            if (c > cbB) p2 = 0.f;
-            if (c + 1 > cbB) p3 = 0.f;
-        }
+        const float p0 = ex2_mufu(fmaf(__uint_as_float(s[4 * g]), sl2, negmA));
+        const float p1 = ex2_mufu(fmaf(__uint_as_float(s[4 * g + 1]), sl2, negmA));
+        const float p2 = ex2_mufu(fmaf(__uint_as_float(s[4 * g + 2]), sl2, negmB));
+        const float p3 = ex2_mufu(fmaf(__uint_as_float(s[4 * g + 3]), sl2, negmB));
         sa0 += p0; sa1 += p1; sb0 += p2; sb1 += p3;
         pk[2 * g] = pack_bf16x2(p0, p1);
         pk[2 * g + 1] = pack_bf16x2(p2, p3);
