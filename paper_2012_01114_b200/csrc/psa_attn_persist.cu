@@ -375,9 +375,12 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                             if (j >= nkv[t]) continue;
                             const uint32_t vc = vbase + j, kc = kbase + j + 1;
                             const bool has_next = j + 1 < nkv[t];
-                            // operand tiles first: these are normally long complete and cost only the poll
-                            if constexpr (!KVS) ok = mbar_wait(&bars.v_full[vc % VST], (vc / VST) & 1, abortp);
-                            if (ok && has_next) ok = mbar_wait(&bars.k_full[kc % KST], (kc / KST) & 1, abortp);
+                            // Operand tiles first.  A probe of a barrier costs this thread 150-200 cycles beside the
+                            // busy softmax warps, so slot 1 does not repeat the ones slot 0 made for the same block.
+                            if constexpr (!KVS)
+                                if (t == 0 || j >= nkv[0]) ok = mbar_wait(&bars.v_full[vc % VST], (vc / VST) & 1, abortp);
+                            if (ok && has_next && (t == 0 || j + 1 >= nkv[0]))
+                                ok = mbar_wait(&bars.k_full[kc % KST], (kc / KST) & 1, abortp);
                             if (ok) ok = mbar_wait(&bars.p_ready[t], (blk0[t] + j) & 1, abortp);
                             if (!ok) break;
                             tc_fence_after();
