@@ -111,8 +111,8 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
             mbar_init(&bars.q_full[t], 1);
             mbar_init(&bars.q_empty[t], 1);
             mbar_init(&bars.s_full[t], 1);
-            mbar_init(&bars.s_free[t], 32 * SOFTMAX_WARPS_PER_TILE);
-            mbar_init(&bars.p_ready[t], 32 * SOFTMAX_WARPS_PER_TILE);
+            mbar_init(&bars.s_free[t], SOFTMAX_WARPS_PER_TILE);       // one arrival per softmax warp
+            mbar_init(&bars.p_ready[t], SOFTMAX_WARPS_PER_TILE);
             mbar_init(&bars.o_done[t], 1);
         }
         for (int s = 0; s < 8; ++s) {
@@ -470,7 +470,8 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                 if (SEP) {
                     // S is in registers: the issuer may overwrite it with the next scores while the exponentials run
                     tc_fence_before();
-                    mbar_arrive(&bars.s_free[t]);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars.s_free[t]);
                 }
                 // ---- pass 1: row maxima of the block, completed inside the quad
                 float bA = -INFINITY, bB = -INFINITY;
@@ -528,7 +529,8 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                 }
                 tc_wait_st();
                 tc_fence_before();
-                mbar_arrive(&bars.p_ready[t]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars.p_ready[t]);      // (one arrival per warp: 32 on one barrier serialise)
             }
             if (!ok) break;
             ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
