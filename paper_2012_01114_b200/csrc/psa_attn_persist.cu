@@ -430,16 +430,23 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
         uint32_t blk = 0;                                       // blocks this tile slot has processed, all items
         bool store_pending = false;                             // a TMA store of this warp may still be reading `stage`
         bool ok = true;
-        for (uint32_t it = 0; ok; ++it) {
-            ok = mbar_wait(&bars.item_full[it & 1], (it >> 1) & 1, abortp);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+        // Takes entry `it` of the item ring: the item's index, -1 at the end of the list, -2 when the wait ran out.
+        auto take_item = [&](uint32_t it) -> int {
+            if (!__all_sync(0xffffffffu, mbar_wait(&bars.item_full[it & 1], (it >> 1) & 1, abortp))) return -2;
             const int idx = item_ring[it & 1];
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars.item_empty[it & 1]);
-            if (idx < 0) break;
-            const CtaWork work = item_work(idx);
-            if (t >= work.ntiles) continue;                     // no rows for this slot in this item
+            return idx;
+        };
+        uint32_t it = 0;
+        int idx = take_item(it++);
+        CtaWork work = idx >= 0 ? item_work(idx) : CtaWork{};
+        while (idx >= 0) {
+            if (t >= work.ntiles) {                             // no rows for this slot in this item
+                idx = take_item(it++);
+                if (idx >= 0) work = item_work(idx);
+                continue;
+            }
             const int b = work.bh / H, h = work.bh - b * H;
             const int It = work.tile0 + t;
             const int nkv = kv_tiles(It, T, scheme);
@@ -533,6 +540,10 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                 if (lane == 0) mbar_arrive(&bars.p_ready[t]);      // (one arrival per warp: 32 on one barrier serialise)
             }
             if (!ok) break;
+            // The next item is taken and decoded now, while the last PV runs, rather than after the epilogue.
+            const int idx_next = take_item(it++);
+            if (idx_next == -2) break;
+            const CtaWork work_next = idx_next >= 0 ? item_work(idx_next) : CtaWork{};
             ok = mbar_wait(&bars.o_done[t], (blk - 1) & 1, abortp);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -568,6 +579,8 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
             // thread of the tile signals only after these reads)
             tc_fence_before();
             ++my_items;
+            idx = idx_next;
+            work = work_next;
         }
         if (store_pending && lane == 0) tma_store_wait_read();   // shared memory may be released; the writes complete on their own
     }
