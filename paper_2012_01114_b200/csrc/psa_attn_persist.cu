@@ -144,8 +144,7 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                 mbar_arrive(&bars.item_full[slot]);
                 if (idx >= nitems) break;
                 const CtaWork work = item_work(idx);
-                // the next item's index is fetched now, long before it is needed
-                const int next = (int)gridDim.x + (int)atomicAdd(&dc->next_item, 1u);
+                int next = -1;
                 const int b = work.bh / H, h = work.bh - b * H;
                 const int nkv0 = kv_tiles(work.tile0, T, scheme);
                 const int nkv1 = work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0;
@@ -183,6 +182,9 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                                         j * TILE, b);
                         ++vc;
                     }
+                    // the next item's index is fetched behind the item's first loads (the atomic's round trip of about
+                    // a thousand cycles would otherwise delay them) and long before it is needed
+                    if (j == 0) next = (int)gridDim.x + (int)atomicAdd(&dc->next_item, 1u);
                 }
                 idx = next;
             }
