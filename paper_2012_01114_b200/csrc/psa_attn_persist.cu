@@ -103,8 +103,6 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        // the counter block of the NEXT call on this workspace is cleared here, off that call's critical path
-        if (blockIdx.x == 0 && dc_next) *dc_next = DeviceCounters{0, 0, 0, 0, 0, 0, 0};
         for (int t = 0; t < 2; ++t) {
             mbar_init(&bars.item_full[t], 1);
             mbar_init(&bars.item_empty[t], item_readers<D>());
@@ -128,6 +126,12 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
     volatile int* abortp = &abort_flag;
+    // Everything above (barriers, TMEM) overlaps the end of the kernel before this one in the stream; global memory
+    // is touched only from here on.
+    grid_launch_dependents();
+    grid_dependency_wait();
+    // the counter block of the NEXT call on this workspace is cleared here, off that call's critical path
+    if (threadIdx.x == 0 && blockIdx.x == 0 && dc_next) *dc_next = DeviceCounters{0, 0, 0, 0, 0, 0, 0};
 
     if (warp == 0) {
         if (lane == 0) {
@@ -614,9 +618,18 @@ int launch_persist(const void* Q, const void* K, const void* V, void* out, int B
     const int grid = (int)(nitems < sm_count ? nitems : sm_count);
     const SchedParams sp = sched_params(n, scheme == PSA_MASKED, B * H, lpt_group(scheme, B * H, n, d),
                                         split == pairs ? 0x7fffffff : (int)split);
-    attn_persist_kernel<D, KVS><<<grid, persist_threads<D>(), Cfg::SMEM, stream>>>(maps, sp, H, scheme, (int)nitems,
-                                                                            scale * LOG2E, dc, dc_next);
-    const cudaError_t e = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(persist_threads<D>());
+    cfg.dynamicSmemBytes = Cfg::SMEM;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // the kernel waits for its predecessor itself
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, attn_persist_kernel<D, KVS>, maps, sp, H, scheme, (int)nitems,
+                                             scale * LOG2E, dc, dc_next);
     if (e != cudaSuccess) { set_cuda_error(e, "attn_persist_kernel launch"); return PSA_ERR_CUDA; }
     return PSA_OK;
 }

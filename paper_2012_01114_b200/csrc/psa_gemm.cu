@@ -162,6 +162,9 @@ gemm_bf16_kernel(const __grid_constant__ GemmMaps maps, int M, int N, int K, int
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
     volatile int* abortp = &abort_flag;
+    // (programmatic dependent launch: the set-up above overlaps the end of the kernel before this one)
+    grid_launch_dependents();
+    grid_dependency_wait();
 
     if (warp == 0 && lane == 0) {
         // ---- TMA producer: k-steps of all this CTA's tiles, numbered g = 0, 1, ... through the ring
@@ -321,8 +324,17 @@ int bf16_project(const void* A, const void* const Bw[3], void* const C[3], int n
     }
     const int ntiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN) * nW;
     const int grid = ntiles < sm_count ? ntiles : sm_count;
-    gemm_bf16_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(maps, M, N, K, nW, static_cast<const uint16_t*>(residual), dc);
-    cudaError_t e = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = GEMM_SMEM;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // the kernel waits for its predecessor itself
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_bf16_kernel, maps, M, N, K, nW, static_cast<const uint16_t*>(residual), dc);
     if (e != cudaSuccess) { set_cuda_error(e, "gemm_bf16_kernel launch"); return PSA_ERR_CUDA; }
     return PSA_OK;
 }

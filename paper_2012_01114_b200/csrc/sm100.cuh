@@ -120,6 +120,14 @@ __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with programmatic stream serialization may become resident while the kernel before it in
+// the stream still runs.  grid_dependency_wait() returns once that kernel has completed and its writes are
+// visible: nothing before it may touch global memory.  grid_launch_dependents() lets the kernel after this one
+// become resident as soon as this grid's CTAs leave room (it still waits, in the same way, for this grid's end).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- proxies / fences
 __device__ __forceinline__ void fence_async_smem() {  // generic-proxy smem writes -> visible to TMA / MMA
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
