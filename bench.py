@@ -41,16 +41,15 @@ L2_FLUSH_BYTES = 256 << 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
 # (attn_persist_kernel_c4_masked_n8192_d128.txt, gemm_and_attn_persist_c3_masked_n1024_d64.txt,
-# attn_persist_kernel_c2_full_n512_d64.txt).  Each figure is tied
-# to the SHA-256 of the sources of the kernel it was measured on; once one of them changes the roofline reports
-# traffic = null.
+# attn_persist_kernel_c2_full_n512_d64.txt, attn_persist_kernel_c5_n256_full_and_masked_d128.txt).  Each figure is tied to the SHA-256 of the sources of the
+# kernel it was measured on; once one of them changes the roofline reports traffic = null.
 NCU_TRAFFIC = {
     "sources": {
-        "psa_attn_persist.cu": "ee15122883433bec99597dda82effe59e574edfea266f1fd984194237566eb60",
-        "psa_softmax.cuh": "083e8baadf062f616a29af748630250fe78a2611c588269cf94d2063a6550cac",
-        "psa_sched.h": "8bfeb6bc6f71007ef2d0044a38a0f5c4d9baf1f9cb73da7f6845232cda8598eb",
-        "psa_gemm.cu": "40aee68e878f71b318a422d7780369c41d78cc0b25fab601b69724467f24b16e",
-        "sm100.cuh": "e7db1e3c78bf7631d027fac7c3a8e2b2db487890b77e0de145ba17783a9ac464"
+        "psa_attn_persist.cu": "da8a086377a45baeace52bc0460e966fc22e3c123c67b20bc15eed72170928fd",
+        "psa_softmax.cuh": "d6f464522774d5fa8e06d7bee0caa46cdbc57e830deef1f6ed5d2fd01c6dae71",
+        "psa_sched.h": "f58d760c07067dcd12ea1f5d021072901f1247fc43730932f168d76ee1dd69aa",
+        "psa_gemm.cu": "5b17be103b323534f4e008f4c4163c602f0856e02554aed95af41983d4b46772",
+        "sm100.cuh": "91d4a36131b303291fee5f482172f435d8c0c5fa8c10e538f005193dd195ab6c"
     },
     "kernel_sources": {
         "attn": ["psa_attn_persist.cu", "psa_softmax.cuh", "psa_sched.h", "sm100.cuh"],
@@ -58,14 +57,21 @@ NCU_TRAFFIC = {
     },
     "traffic_bytes": {
         "c4": {
-            "attn": 592754176
+            "attn": 594941696
         },
         "c3": {
-            "attn": 37837824,
-            "proj": 16199936
+            "attn": 38173440,
+            "proj": 16342272
         },
         "c2": {
-            "attn": 18939904
+            "attn": 19240192,
+            "proj": 9854464
+        },
+        "c5-n256-full": {
+            "attn": 1045856768
+        },
+        "c5-n256-masked": {
+            "attn": 1046352896
         }
     }
 }

@@ -24,8 +24,8 @@
  *   - `scale` multiplies the phase-1 dot product (Eq. 1 has no 1/sqrt(d); scale = 1 gives
  *     the literal equation).
  *   - exp is evaluated on w' minus the row maximum; mathematically equal to Eq. 2.
- *   - the main diagonal is kept by the mask (Sec. 5.1: "main diagonal and the lower
- *     triangular part").
+ *   - the main diagonal is kept by the mask (Sec. 5.1 lists the diagonal among the weights that
+ *     remain, together with everything below it).
  *
  * Counters are incremented inside the loops that do the work, so they are a census of
  * the operations performed, not a formula.
