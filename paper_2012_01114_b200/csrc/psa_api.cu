@@ -134,7 +134,9 @@ void useful_counts(int batch, int heads, int n, int d_model, int d_k, int scheme
 int run_layer(Context& cx, const void* X, const void* Wq, const void* Wk, const void* Wv, const void* Q, const void* K,
               const void* V, int batch, int heads, int n, int d_model, int d_k, int scheme, int dtype, void* out,
               cudaStream_t stream, bool with_proj, char* ws, const WsLayout& L) {
-    const bool turns = dtype == PSA_BF16 && scheme != PSA_SYMMETRIC;   // the path whose last kernel clears the other block
+    // the paths whose last kernel clears the other counter block: the fused bf16 kernel and the one-launch fp32 layer
+    const bool fused_f32 = with_proj && dtype == PSA_F32 && f32_fused_fits(n, d_model, d_k, scheme);
+    const bool turns = (dtype == PSA_BF16 && scheme != PSA_SYMMETRIC) || fused_f32;
     int block = 0;
     cudaError_t e = cudaSuccess;
     if (turns && cx.clean_ws == ws) {
@@ -158,13 +160,15 @@ int run_layer(Context& cx, const void* X, const void* Wq, const void* Wk, const 
         ~EventTail() { if (ev) cudaEventRecord(ev[2], st); }
     } tail{pev, stream};
     if (pev) cudaEventRecord(pev[0], stream);
-    if (with_proj && dtype == PSA_F32 && f32_fused_fits(n, d_model, d_k, scheme)) {
+    if (fused_f32) {
         // a small fp32 layer runs as one launch; q, k, v never leave shared memory
         if (pev) cudaEventRecord(pev[1], stream);
         e = f32_fused_layer(static_cast<const float*>(X), static_cast<const float*>(Wq), static_cast<const float*>(Wk),
                             static_cast<const float*>(Wv), static_cast<float*>(out), batch, heads, n, d_model, d_k, scale,
-                            scheme, dc, stream);
+                            scheme, dc, dc_next, stream);
         if (e != cudaSuccess) { set_cuda_error(e, "f32_fused_layer"); return PSA_ERR_CUDA; }
+        cx.clean_ws = ws;               // the other block will be clear once this call has run
+        cx.next_block = block ^ 1;
         return PSA_OK;
     }
     if (with_proj) {

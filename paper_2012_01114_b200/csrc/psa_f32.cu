@@ -2,6 +2,8 @@
 // scheme does not need is never computed (paper Sec. 4.1, 5.1), so issued MACs equal the paper's
 // element counts (Sec. 3.2, 4.2, 5.2).  Meant for small problems and as the full-precision path;
 // the throughput path is the bf16 tensor-core one.
+#include <cooperative_groups.h>
+
 #include "psa_internal.h"
 
 namespace psa {
@@ -168,9 +170,11 @@ __host__ __device__ inline FusedLayout fused_layout(int n, int D, int d, int nW)
 __global__ void __launch_bounds__(FS_THREADS, 1)
 f32_fused_layer_kernel(const float* __restrict__ X, const float* __restrict__ Wq, const float* __restrict__ Wk,
                        const float* __restrict__ Wv, float* __restrict__ out, int n, int H, int D, int d, float scale,
-                       int scheme, DeviceCounters* dc) {
+                       int scheme, DeviceCounters* dc, DeviceCounters* dc_next) {
     extern __shared__ float4 fs_smem4[];
     float* sm = reinterpret_cast<float*>(fs_smem4);
+    // the counter block of the NEXT call on this workspace is cleared here, off that call's critical path
+    if (blockIdx.x == 0 && threadIdx.x == 0 && dc_next) *dc_next = DeviceCounters{0, 0, 0, 0, 0, 0, 0};
     const int nW = scheme == PSA_SYMMETRIC ? 1 : 3;
     const FusedLayout L = fused_layout(n, D, d, nW);
     float* xs = sm + L.xs; float* ws = sm + L.ws; float* qt = sm + L.qt; float* kt = sm + L.kt; float* vs = sm + L.vs;
@@ -360,6 +364,185 @@ f32_fused_layer_kernel(const float* __restrict__ X, const float* __restrict__ Wq
     if (tid == 0) atomicAdd(&dc->proj_macs, (unsigned long long)nW * n * D * d);
 }
 
+// Asynchronous copies global -> shared (4 and 16 bytes) and the wait for all of a thread's copies.
+__device__ __forceinline__ void cp_async4(float* dst, const float* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async16(float* dst, const float* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// The same layer spread over a cluster of C CTAs (FULL and MASKED): 4-row tiles are dealt to the CTAs in turn (tile ti
+// belongs to CTA ti % C, which balances the masked scheme's growing rows), each CTA projects q, k, v of its own rows,
+// the CTAs read one another's k and v through distributed shared memory, and each finishes phases 1-3 for its rows.
+// A layer of one head then occupies C SMs instead of one.  Tasks are one row by four columns, so that the few rows a
+// CTA owns still spread over its threads; the census is element-exact as above.
+__global__ void __launch_bounds__(FS_THREADS, 1)
+f32_fused_cluster_kernel(const float* __restrict__ X, const float* __restrict__ Wq, const float* __restrict__ Wk,
+                         const float* __restrict__ Wv, float* __restrict__ out, int n, int H, int D, int d, float scale,
+                         int scheme, DeviceCounters* dc, DeviceCounters* dc_next) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int C = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+    extern __shared__ float4 fs_smem4[];
+    float* sm = reinterpret_cast<float*>(fs_smem4);
+    const FusedLayout L = fused_layout(n, D, d, 3);
+    float* xs = sm + L.xs; float* ws = sm + L.ws; float* qt = sm + L.qt; float* kt = sm + L.kt; float* vs = sm + L.vs;
+    float* S = sm + L.sm; float* rinv = sm + L.rinv;
+    const int head = blockIdx.x / C, b = head / H, h = head - b * H;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool masked = scheme == PSA_MASKED;
+    const size_t HD = (size_t)H * d;
+    const int tn = (n + 3) / 4, tc = d / 4;
+    const int own_tiles = rank < tn ? (tn - rank + C - 1) / C : 0;     // tiles rank, rank + C, ...
+    const int own_rows = own_tiles * 4;                                // (the last tile's rows beyond n are skipped)
+    auto own_row = [&](int lr) { return 4 * (rank + (lr >> 2) * C) + (lr & 3); };     // local row -> row of the head
+    unsigned long long qk = 0, pv = 0, ex = 0, pj = 0;
+    if (blockIdx.x == 0 && tid == 0 && dc_next) *dc_next = DeviceCounters{0, 0, 0, 0, 0, 0, 0};
+
+    // ---- stage this CTA's rows of X[b] and the head's columns of the three projection matrices: asynchronous copies
+    // straight into shared memory, all in flight at once (a layer this small lives on the latency of its first loads)
+    {
+        const float* xb = X + (size_t)b * n * D;
+        for (int t = tid; t < own_rows * D; t += FS_THREADS) {
+            const int lr = t / D, k = t - lr * D, i = own_row(lr);
+            if (i < n) cp_async4(xs + i * L.xs_ld + k, xb + (size_t)i * D + k);
+        }
+        const int d4 = d / 4;
+        for (int t = tid; t < 3 * D * d4; t += FS_THREADS) {
+            const int w = t / (D * d4), rem = t - w * D * d4, k = rem / d4, c4 = rem - k * d4;
+            const float* W = (w == 0 ? Wq : (w == 1 ? Wk : Wv)) + (size_t)h * d;
+            cp_async16(ws + (size_t)w * D * d + (size_t)k * d + 4 * c4, W + (size_t)k * HD + 4 * c4);
+        }
+        cp_async_wait_all();
+    }
+    __syncthreads();
+
+    // ---- projections (Sec. 3.1) of the own rows: one row by four columns per task
+    for (int t = tid; t < 3 * own_rows * tc; t += FS_THREADS) {
+        const int w = t / (own_rows * tc), rem = t - w * own_rows * tc;
+        const int lr = rem / tc, c0 = (rem - lr * tc) * 4, i = own_row(lr);
+        if (i >= n) continue;
+        const float* wp = ws + (size_t)w * D * d + c0;
+        const float* xr = xs + (size_t)i * L.xs_ld;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+        for (int k = 0; k < D; ++k) {
+            const float4 wv = *reinterpret_cast<const float4*>(wp + (size_t)k * d);
+            const float x = xr[k];
+            acc.x = fmaf(x, wv.x, acc.x); acc.y = fmaf(x, wv.y, acc.y); acc.z = fmaf(x, wv.z, acc.z); acc.w = fmaf(x, wv.w, acc.w);
+        }
+        if (w < 2) {
+            float* dst = (w == 0 ? qt : kt) + i;
+            dst[(size_t)(c0 + 0) * L.t_ld] = acc.x; dst[(size_t)(c0 + 1) * L.t_ld] = acc.y;
+            dst[(size_t)(c0 + 2) * L.t_ld] = acc.z; dst[(size_t)(c0 + 3) * L.t_ld] = acc.w;
+        } else {
+            *reinterpret_cast<float4*>(vs + (size_t)i * L.ds + c0) = acc;
+        }
+        pj += 4ull * D;
+    }
+    cluster.sync();           // every CTA's k and v rows are in its shared memory
+
+    // ---- k and v of the other CTAs' rows, one 4-row tile (16 bytes of a transposed k component; a row of v) at a time
+    for (int t = tid; t < d * tn; t += FS_THREADS) {
+        const int c = t / tn, ti = t - c * tn, owner = ti % C;
+        if (owner == rank) continue;
+        const float* src = cluster.map_shared_rank(kt, owner);
+        *reinterpret_cast<float4*>(kt + (size_t)c * L.t_ld + 4 * ti) = *reinterpret_cast<const float4*>(src + (size_t)c * L.t_ld + 4 * ti);
+    }
+    for (int t = tid; t < n * tc; t += FS_THREADS) {
+        const int i = t / tc, c0 = (t - i * tc) * 4, owner = (i >> 2) % C;
+        if (owner == rank) continue;
+        const float* src = cluster.map_shared_rank(vs, owner);
+        *reinterpret_cast<float4*>(vs + (size_t)i * L.ds + c0) = *reinterpret_cast<const float4*>(src + (size_t)i * L.ds + c0);
+    }
+    cluster.sync();           // no CTA reads another's shared memory from here on
+
+    // ---- phase 1 (Eq. 1) for the own rows: S_ij = scale q_i . k_j, one row by four keys per task; a key beyond the
+    // row's last kept one (masked: j > i; the edge: j >= n) is never computed
+    for (int t = tid; t < own_rows * tn; t += FS_THREADS) {
+        const int lr = t / tn, j0 = (t - lr * tn) * 4, i = own_row(lr);
+        if (i >= n) continue;
+        const int jlast = masked ? i : n - 1;
+        if (j0 > jlast) continue;
+        const int cnt = min(4, jlast - j0 + 1);                   // keys j0 .. j0 + cnt - 1 are kept
+        const float* qp = qt + i;
+        const float* kp = kt + j0;
+        float* row = S + (size_t)i * L.s_ld + j0;
+        if (cnt == 4) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+            for (int c = 0; c < d; ++c) {
+                const float q = qp[(size_t)c * L.t_ld];
+                const float4 k4 = *reinterpret_cast<const float4*>(kp + (size_t)c * L.t_ld);
+                acc.x = fmaf(q, k4.x, acc.x); acc.y = fmaf(q, k4.y, acc.y); acc.z = fmaf(q, k4.z, acc.z); acc.w = fmaf(q, k4.w, acc.w);
+            }
+            row[0] = acc.x * scale; row[1] = acc.y * scale; row[2] = acc.z * scale; row[3] = acc.w * scale;
+        } else {
+            for (int u = 0; u < cnt; ++u) {
+                float acc = 0.f;
+                for (int c = 0; c < d; ++c) acc = fmaf(qp[(size_t)c * L.t_ld], kp[(size_t)c * L.t_ld + u], acc);
+                row[u] = acc * scale;
+            }
+        }
+        qk += (unsigned long long)cnt * d;
+    }
+    __syncthreads();
+
+    // ---- phase 2 (Eq. 2): one warp per own row; the division is applied to the output row
+    for (int lr = warp; lr < own_rows; lr += FS_THREADS / 32) {
+        const int i = own_row(lr);
+        if (i >= n) continue;
+        const int jend = masked ? i + 1 : n;
+        float* row = S + (size_t)i * L.s_ld;
+        float mx = -INFINITY;
+        for (int j = lane; j < jend; j += 32) mx = fmaxf(mx, row[j]);
+        for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        float sum = 0.f;
+        for (int j = lane; j < jend; j += 32) {
+            const float e = expf(row[j] - mx);
+            row[j] = e;
+            sum += e;
+        }
+        for (int off = 16; off; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        if (lane == 0) { rinv[i] = 1.f / sum; ex += (unsigned long long)jend; }
+    }
+    __syncthreads();
+
+    // ---- phase 3 (Eq. 3): y_i = sum_j w_ij v_j over the kept weights, four output components per task
+    for (int t = tid; t < own_rows * tc; t += FS_THREADS) {
+        const int lr = t / tc, c0 = (t - lr * tc) * 4, i = own_row(lr);
+        if (i >= n) continue;
+        const int jend = masked ? i + 1 : n;
+        const float* row = S + (size_t)i * L.s_ld;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+        for (int j = 0; j < jend; ++j) {
+            const float w = row[j];
+            const float4 v = *reinterpret_cast<const float4*>(vs + (size_t)j * L.ds + c0);
+            acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y); acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+        }
+        const float r = rinv[i];
+        *reinterpret_cast<float4*>(out + ((size_t)b * n + i) * HD + (size_t)h * d + c0) = make_float4(acc.x * r, acc.y * r, acc.z * r, acc.w * r);
+        pv += 4ull * jend;
+    }
+
+    // ---- census
+    for (int off = 16; off; off >>= 1) {
+        qk += __shfl_xor_sync(0xffffffffu, qk, off);
+        pv += __shfl_xor_sync(0xffffffffu, pv, off);
+        ex += __shfl_xor_sync(0xffffffffu, ex, off);
+        pj += __shfl_xor_sync(0xffffffffu, pj, off);
+    }
+    if (lane == 0) {
+        if (qk) atomicAdd(&dc->qk_macs, qk);
+        if (pv) atomicAdd(&dc->pv_macs, pv);
+        if (ex) atomicAdd(&dc->exps, ex);
+        if (pj) atomicAdd(&dc->proj_macs, pj);
+    }
+}
+
 size_t attn_smem_bytes(int n, int d) {
     return sizeof(float) * ((size_t)KEY_TILE * (d + 1) + (size_t)ROWS_PER_BLOCK * d + (size_t)ROWS_PER_BLOCK * n);
 }
@@ -378,18 +561,47 @@ bool f32_fused_fits(int n, int D, int d, int scheme) {
     return fused_layout(n, D, d, scheme == PSA_SYMMETRIC ? 1 : 3).total <= (size_t)FS_MAX_FLOATS;
 }
 
+// Heads few enough that one CTA each would leave most SMs idle are spread over clusters of up to 8 CTAs.
+int f32_fused_cluster_size(int B, int H, int n, int scheme) {
+    if (scheme == PSA_SYMMETRIC || B * H > 32) return 1;      // (the symmetric scheme's mirrored store crosses row owners)
+    const int tn = (n + 3) / 4;
+    int c = 1;
+    while (c < 8 && 2 * c <= tn) c *= 2;
+    return c;
+}
+
 cudaError_t f32_fused_layer(const float* X, const float* Wq, const float* Wk, const float* Wv, float* out, int B, int H,
-                            int n, int D, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream) {
+                            int n, int D, int d, float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next,
+                            cudaStream_t stream) {
     static DeviceSetup setup;
     if (device_setup(&setup, [] {
-            return cudaFuncSetAttribute(f32_fused_layer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaError_t e = cudaFuncSetAttribute(f32_fused_layer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 FS_MAX_FLOATS * (int)sizeof(float));
+            if (e != cudaSuccess) return e;
+            return cudaFuncSetAttribute(f32_fused_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         FS_MAX_FLOATS * (int)sizeof(float));
         }, "fp32 fused layer set-up") <= 0)
         return cudaErrorUnknown;
+    const int C = f32_fused_cluster_size(B, H, n, scheme);
+    if (C > 1) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(B * H * C);
+        cfg.blockDim = dim3(FS_THREADS);
+        cfg.dynamicSmemBytes = fused_layout(n, D, d, 3).total * sizeof(float);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = C;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, f32_fused_cluster_kernel, X, Wq, Wk, Wv, out, n, H, D, d, scale, scheme, dc, dc_next);
+    }
     const size_t smem = fused_layout(n, D, d, scheme == PSA_SYMMETRIC ? 1 : 3).total * sizeof(float);
     f32_fused_layer_kernel<<<B * H, FS_THREADS, smem, stream>>>(X, Wq, scheme == PSA_SYMMETRIC ? Wq : Wk,
                                                                scheme == PSA_SYMMETRIC ? Wq : Wv, out, n, H, D, d, scale,
-                                                               scheme, dc);
+                                                               scheme, dc, dc_next);
     return cudaGetLastError();
 }
 

@@ -34,7 +34,8 @@ cudaError_t f32_attention(const float* Q, const float* K, const float* V, float*
 // f32_fused_fits says whether a shape qualifies.  X [B, n, D], W* [D, H*d] (Wk, Wv ignored for PSA_SYMMETRIC).
 bool f32_fused_fits(int n, int D, int d, int scheme);
 cudaError_t f32_fused_layer(const float* X, const float* Wq, const float* Wk, const float* Wv, float* out, int B, int H,
-                            int n, int D, int d, float scale, int scheme, DeviceCounters* dc, cudaStream_t stream);
+                            int n, int D, int d, float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next,
+                            cudaStream_t stream);   // (dc_next, if given, is cleared by the kernel for the next call)
 
 // ---- bf16 tcgen05 path (psa_gemm.cu, psa_attn.cu) ----
 // C[w][M, N] = A[M, K] * Bw[w][K, N] (+ residual[M, N], bf16, may be null), bf16 row-major, fp32 accumulation.
