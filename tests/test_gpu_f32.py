@@ -51,6 +51,26 @@ def test_layer_shapes_and_schemes(scheme, B, H, n, D, d):
     _check_counts(cnt, (1 if sym else 3) * B * n * D * H * d)
 
 
+# Small layers run as one launch; with at most 32 heads the FULL and MASKED schemes spread a head over a cluster of
+# 1, 2, 4 or 8 CTAs (the largest power of two that leaves every CTA a 4-row tile).  The shapes walk those cluster sizes,
+# ragged last tiles, the switch back to one CTA per head at 33 heads, and d_k at both ends of the range.
+@pytest.mark.parametrize("scheme", [oracle.FULL, oracle.MASKED])
+@pytest.mark.parametrize("B,H,n,D,d", [(1, 1, 3, 16, 8), (1, 1, 8, 16, 8), (1, 2, 13, 24, 4), (2, 2, 17, 40, 12),
+                                       (1, 1, 31, 64, 64), (1, 3, 33, 20, 128), (4, 8, 64, 64, 32), (3, 11, 45, 32, 16),
+                                       (1, 1, 130, 48, 64), (1, 1, 256, 32, 32)])
+def test_small_layers_on_clusters(scheme, B, H, n, D, d):
+    rng = np.random.default_rng(1000 * n + d + B)
+    X = (rng.standard_normal((B, n, D)) * 0.5).astype(np.float32)
+    Ws = [(rng.standard_normal((D, H * d)) / np.sqrt(D)).astype(np.float32) for _ in range(3)]
+    ref, cnt = oracle.attention_layer(X, Ws[0], Ws[1], Ws[2], H, scheme)
+    dev = [_dev(X)] + [_dev(w) for w in Ws]
+    for call in range(3):       # the two counter blocks of the workspace are used in turn: every call starts from zero
+        out = binding.psa_attention_f32(dev[0], dev[1], dev[2], dev[3], H, scheme)
+        err = np.abs(out.cpu().numpy().astype(np.float64) - ref).max()
+        assert err <= TOL_F32, (call, err)
+        _check_counts(cnt, 3 * B * n * D * H * d)
+
+
 @pytest.mark.parametrize("scheme", [oracle.FULL, oracle.SYMMETRIC, oracle.MASKED])
 def test_core_entry(scheme):
     rng = np.random.default_rng(5)
