@@ -45,7 +45,7 @@ L2_FLUSH_BYTES = 256 << 20
 # kernel it was measured on; once one of them changes the roofline reports traffic = null.
 NCU_TRAFFIC = {
     "sources": {
-        "psa_attn_persist.cu": "da8a086377a45baeace52bc0460e966fc22e3c123c67b20bc15eed72170928fd",
+        "psa_attn_persist.cu": "1545c1ceb149fdb1acc7efc46fadbd9f8291f9393da26d70c70aeb3031511551",
         "psa_softmax.cuh": "d6f464522774d5fa8e06d7bee0caa46cdbc57e830deef1f6ed5d2fd01c6dae71",
         "psa_sched.h": "f58d760c07067dcd12ea1f5d021072901f1247fc43730932f168d76ee1dd69aa",
         "psa_gemm.cu": "5b17be103b323534f4e008f4c4163c602f0856e02554aed95af41983d4b46772",

@@ -74,8 +74,8 @@ typedef struct {
  * Projections + attention, bf16 in / bf16 out, fp32 accumulation (paper Sec. 3.1 then Eq. 1-3).
  *   X, Wq, Wk, Wv, out   device, bf16, layouts above.
  *   PSA_SYMMETRIC: q = k = v = X*Wq (paper Sec. 4.1); Wk and Wv must be NULL or equal to Wq.
- * Supported: d_k any multiple of 8 up to 128 (the kernels work on heads of 64 or 128 columns; a shorter head is
- * zero-padded by the tile loads, and the census counts the padded width as issued); any n >= 1 (a last block of
+ * Supported: d_k any multiple of 8 up to 256 (PSA_SYMMETRIC: up to 128).  The kernels work on heads of 64, 128 or
+ * 256 columns; a shorter head is zero-padded by the tile loads, and the census counts the padded width as issued; any n >= 1 (a last block of
  * fewer than 128 vectors is zero-filled and its keys carry no weight); d_model and heads*d_k multiples of 64.
  * Needs a workspace of psa_workspace_bytes(...) (grown on demand, see psa_set_workspace).
  */

@@ -196,7 +196,7 @@ def psa_attention_core_host(Q, K, V, scheme, out, stream=None):
     rc = lib().psa_attention_core_host(_ptr(Q), _ptr(K), _ptr(V), B, H, n, d, int(scheme), code, _ptr(out),
                                        _stream(stream))
     if rc != OK:
-        raise PsaError(rc, "psa_attention_core_host", "psa_attention_block_residual")
+        raise PsaError(rc, "psa_attention_core_host")
     return out
 
 
@@ -223,7 +223,7 @@ def psa_measure_pipe_rates(stream=None) -> dict:
     r = PipeRates()
     rc = lib().psa_measure_pipe_rates(ctypes.byref(r), _stream(stream))
     if rc != OK:
-        raise PsaError(rc, "psa_measure_pipe_rates", "psa_attention_core_host", "psa_attention_block_residual")
+        raise PsaError(rc, "psa_measure_pipe_rates")
     return {k: getattr(r, k) for k, _ in r._fields_}
 
 
@@ -239,7 +239,7 @@ def psa_last_rescales(stream=None) -> int:
     v = ctypes.c_uint64()
     rc = lib().psa_last_rescales(_stream(stream), ctypes.byref(v))
     if rc != OK:
-        raise PsaError(rc, "psa_last_rescales", "psa_selftest_wait_expiry", "psa_measure_pipe_rates", "psa_attention_core_host", "psa_attention_block_residual")
+        raise PsaError(rc, "psa_last_rescales")
     return int(v.value)
 
 

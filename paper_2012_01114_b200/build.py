@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpsa.so")
-SOURCES = ["psa_api.cu", "psa_f32.cu", "psa_gemm.cu", "psa_attn.cu", "psa_attn_persist.cu", "psa_noalloc.cu", "psa_selftest.cu", "psa_pipes.cu"]
+SOURCES = ["psa_api.cu", "psa_f32.cu", "psa_gemm.cu", "psa_attn.cu", "psa_attn_persist.cu", "psa_attn_wide.cu", "psa_noalloc.cu", "psa_selftest.cu", "psa_pipes.cu"]
 
 
 def _sources():

@@ -61,7 +61,8 @@ int check_shape(int batch, int heads, int n, int d_model, int d_k, int scheme, i
         return PSA_ERR_SHAPE;
     if ((long long)batch * n > 0x7fffffffLL || (long long)heads * d_k > 0x7fffffffLL) return PSA_ERR_SHAPE;
     if (dtype == PSA_BF16) {
-        if (d_k < 8 || d_k > 128 || d_k % 8 != 0) return PSA_ERR_UNSUPPORTED;
+        // heads of up to 256 columns for the full and masked schemes; the symmetric scheme's kernels stop at 128
+        if (d_k < 8 || d_k > (scheme == PSA_SYMMETRIC ? 128 : 256) || d_k % 8 != 0) return PSA_ERR_UNSUPPORTED;
         if (with_proj && (d_model % 64 != 0)) return PSA_ERR_UNSUPPORTED;
     } else {
         if (n > 1024 || d_k > 128) return PSA_ERR_UNSUPPORTED;
@@ -136,7 +137,7 @@ int run_layer(Context& cx, const void* X, const void* Wq, const void* Wk, const 
               cudaStream_t stream, bool with_proj, char* ws, const WsLayout& L) {
     // the paths whose last kernel clears the other counter block: the fused bf16 kernel and the one-launch fp32 layer
     const bool fused_f32 = with_proj && dtype == PSA_F32 && f32_fused_fits(n, d_model, d_k, scheme);
-    const bool turns = (dtype == PSA_BF16 && scheme != PSA_SYMMETRIC) || fused_f32;
+    const bool turns = (dtype == PSA_BF16 && scheme != PSA_SYMMETRIC && d_k <= 128) || fused_f32;
     int block = 0;
     cudaError_t e = cudaSuccess;
     if (turns && cx.clean_ws == ws) {
@@ -440,9 +441,9 @@ int psa_skip_count(int batch, int heads, int n, int d_model, int d_k, int scheme
     // pairs of a launch out as single row tiles, split_point in psa_sched.h, those are the same row tiles with the
     // same block lists taken one at a time: the census does not depend on the grouping.)
     const int T = row_tiles(n);
-    // (a head size below the 64 or 128 columns the kernels work with is zero-padded by the loads: the padded
+    // (a head size below the 64, 128 or 256 columns the kernels work with is zero-padded by the loads: the padded
     // width is what the tensor core is issued)
-    const uint64_t block_macs = (uint64_t)TILE * TILE * (d_k <= 64 ? 64 : 128);
+    const uint64_t block_macs = (uint64_t)TILE * TILE * (d_k <= 64 ? 64 : (d_k <= 128 ? 128 : 256));
     uint64_t qk_blocks = 0, pv_blocks = 0, exps = 0;
     const int P = ctas_per_head(n);
     for (int cta = 0; cta < P; ++cta) {  // every head has the same list

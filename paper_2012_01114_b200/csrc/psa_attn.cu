@@ -460,6 +460,7 @@ size_t bf16_symmetric_scratch_bytes(int B, int H, int n) {
 
 int bf16_attention(const void* Q, const void* K, const void* V, void* out, float* S, size_t s_bytes, int B, int H,
                    int n, int d, float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream) {
+    if (scheme != PSA_SYMMETRIC && d > 128) return bf16_attention_wide(Q, K, V, out, B, H, n, d, scale, scheme, dc, stream);
     if (scheme != PSA_SYMMETRIC) return bf16_attention_persist(Q, K, V, out, B, H, n, d, scale, scheme, dc, dc_next, stream);
     if (!S || s_bytes < bf16_symmetric_scratch_bytes(B, H, n)) return PSA_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(S) & 15u) != 0) return PSA_ERR_ALIGN;

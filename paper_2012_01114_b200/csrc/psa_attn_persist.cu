@@ -3,9 +3,9 @@
 // matrix, as ONE persistent kernel: a CTA per SM walks the tile scheduler's work list.
 //
 //   phase 1  S = Q K^T            tcgen05 MMA, operands staged by TMA, accumulator in TMEM
-//   phase 2  softmax              two threads per query row (64 columns each) read S from TMEM, keep a
+//   phase 2  softmax              a warp reads 16 query rows of S from TMEM in the quad layout, keeps a
 //                                 running row maximum m and row sum l (the division of Eq. 2 is
-//                                 applied once to the output row), write P = exp2(..) as bf16 to TMEM
+//                                 applied once to the output row), writes P = exp2(..) as bf16 to TMEM
 //   phase 3  O += P V             tcgen05 MMA with P read from TMEM and V (row-major = MN-major) from
 //                                 shared memory, accumulator O in TMEM
 //
@@ -24,12 +24,10 @@
 //
 // CTA layout (576 threads; 608 at d = 64): warp 0 = scheduler + TMA producer, warp 1 = MMA issuer, warps 2-9 =
 // softmax and epilogue of row tile 0, warps 10-17 = the same for row tile 1 (d = 64: warp 18 = MMA issuer of row
-// tile 1, warp 1 that of row tile 0).  Within a tile's eight warps,
-// warp pairs (w, w+4) share a TMEM lane quarter (32 rows) and split the 128 columns of S in halves;
-// the pair agrees on the row maximum through shared memory.
-// TMEM columns, d = 128: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_t (bf16, two per
-// column) overlays S_t: keys 0-63 at S_t columns [0,32), keys 64-127 at [64,96), each written by the
-// thread that owns that half of the row.  d = 64: S0 S1 | P0 P1 [256,384) | O0 O1 [384,512): P has
+// tile 1, warp 1 that of row tile 0).  Within a tile's eight warps, warp w owns the 16 rows
+// 32 (w % 4) + 16 (w / 4) .. + 15 (a warp may touch only its own quarter of the TMEM lanes) and all 128 columns of S.
+// TMEM columns, d = 128: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_t (bf16, two keys per
+// column) overlays the first 64 columns of S_t.  d = 64: S0 S1 | P0 P1 [256,384) | O0 O1 [384,512): P has
 // its own columns, so S of the next key block is computed while the softmax of the current one runs.
 #include "psa_internal.h"
 #include "psa_sched.h"

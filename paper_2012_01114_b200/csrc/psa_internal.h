@@ -49,6 +49,9 @@ int bf16_attention(const void* Q, const void* K, const void* V, void* out, float
                    int H, int n, int d, float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next,
                    cudaStream_t stream);
 size_t bf16_symmetric_scratch_bytes(int B, int H, int n);
+// PSA_FULL and PSA_MASKED for 128 < d <= 256: one row tile per CTA (psa_attn_wide.cu).
+int bf16_attention_wide(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, int d, float scale,
+                        int scheme, DeviceCounters* dc, cudaStream_t stream);
 // The persistent fused kernel behind bf16_attention for PSA_FULL and PSA_MASKED (psa_attn_persist.cu).
 int bf16_attention_persist(const void* Q, const void* K, const void* V, void* out, int B, int H, int n, int d,
                            float scale, int scheme, DeviceCounters* dc, DeviceCounters* dc_next, cudaStream_t stream);

@@ -76,7 +76,9 @@ def test_argument_errors_launch_nothing(lib):
     assert lib.psa_skip_count(1, 1, 100, 0, 64, 0, binding.BF16, ctypes.byref(c)) == binding.OK      # ragged n is fine
     assert lib.psa_skip_count(1, 1, 128, 100, 64, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED  # d_model % 64
     assert lib.psa_skip_count(1, 1, 128, 0, 100, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED   # d_k % 8
-    assert lib.psa_skip_count(1, 1, 128, 0, 256, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED   # d_k > 128
+    assert lib.psa_skip_count(1, 1, 128, 0, 256, 0, binding.BF16, ctypes.byref(c)) == binding.OK               # up to 256 columns
+    assert lib.psa_skip_count(1, 1, 128, 0, 264, 0, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED   # d_k > 256
+    assert lib.psa_skip_count(1, 1, 128, 0, 256, 1, binding.BF16, ctypes.byref(c)) == binding.ERR_UNSUPPORTED   # symmetric: up to 128
     assert lib.psa_skip_count(1, 1, 128, 0, 96, 0, binding.BF16, ctypes.byref(c)) == binding.OK
     assert c.qk_macs == 128 * 128 * 128 and c.useful_qk_macs == 128 * 128 * 96    # issued at the padded width of 128
     assert lib.psa_skip_count(1, 1, 2048, 0, 64, 0, binding.F32, ctypes.byref(c)) == binding.ERR_UNSUPPORTED
