@@ -48,8 +48,8 @@ NCU_TRAFFIC = {
         "psa_attn_persist.cu": "1545c1ceb149fdb1acc7efc46fadbd9f8291f9393da26d70c70aeb3031511551",
         "psa_softmax.cuh": "d6f464522774d5fa8e06d7bee0caa46cdbc57e830deef1f6ed5d2fd01c6dae71",
         "psa_sched.h": "f58d760c07067dcd12ea1f5d021072901f1247fc43730932f168d76ee1dd69aa",
-        "psa_gemm.cu": "5b17be103b323534f4e008f4c4163c602f0856e02554aed95af41983d4b46772",
-        "sm100.cuh": "91d4a36131b303291fee5f482172f435d8c0c5fa8c10e538f005193dd195ab6c"
+        "psa_gemm.cu": "aa5a23d2e10a143ef90f2ed14bea1e072da286f79f0fd239b70736824174756c",
+        "sm100.cuh": "2cc54c0ff8d920951dbbb97cef53e6b0fc9bd7d43d4002998c5a93069abcd23c"
     },
     "kernel_sources": {
         "attn": ["psa_attn_persist.cu", "psa_softmax.cuh", "psa_sched.h", "sm100.cuh"],

@@ -60,25 +60,6 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uin
     return true;
 }
 
-bool make_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t batch, uint64_t n, uint64_t cols,
-                             uint32_t box_rows) {
-    if (!resolve_encode()) return false;
-    cuuint64_t dims[3] = {cols, n, batch};
-    cuuint64_t strides[2] = {cols * 2, n * cols * 2};
-    cuuint32_t box[3] = {64, box_rows, 1};
-    cuuint32_t es[3] = {1, 1, 1};
-    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-        char msg[96];
-        snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled (3-D) failed with CUresult %d", (int)r);
-        set_error_text(msg);
-        return false;
-    }
-    return true;
-}
-
 bool make_tensor_map_bf16_4d(CUtensorMap* map, const void* base, uint64_t batch, uint64_t n, uint64_t heads, uint64_t d,
                              uint32_t box_rows) {
     if (!resolve_encode()) return false;

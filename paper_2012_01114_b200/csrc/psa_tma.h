@@ -13,11 +13,6 @@ namespace psa {
 bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_bytes,
                           uint32_t box_rows, uint32_t box_cols);
 
-// Tensor map over a [batch, n, cols] bf16 tensor (dense): boxes are [1 x box_rows x 64 columns]; rows beyond n
-// are out of bounds of the map (zero fill on load, dropped on store).
-bool make_tensor_map_bf16_3d(CUtensorMap* map, const void* base, uint64_t batch, uint64_t n, uint64_t cols,
-                             uint32_t box_rows);
-
 // Tensor map over a [batch, n, heads, d] bf16 tensor (dense, d a multiple of 8): boxes are [1 x box_rows x 1 head x
 // 64 elements]; elements beyond d and rows beyond n are out of bounds of the map (zero fill on load, dropped on store).
 bool make_tensor_map_bf16_4d(CUtensorMap* map, const void* base, uint64_t batch, uint64_t n, uint64_t heads, uint64_t d,

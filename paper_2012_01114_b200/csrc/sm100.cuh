@@ -60,18 +60,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// One probe that never suspends: true when the phase with the given parity has completed.
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
 // Bounded wait for the phase with the given parity to complete.  `abort_flag` lives in shared
 // memory; any thread that gives up (after `limit_ns`) sets it and every other waiter leaves at its next poll.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
@@ -137,10 +125,7 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// ---------------------------------------------------------------- TMA (tiled, 2-D, no cluster features)
-__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
-}
+// ---------------------------------------------------------------- TMA (tiled, no cluster features)
 // x = innermost (element) coordinate, must be a multiple of 8 for 16-bit elements; y = row.
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int x, int y) {
     asm volatile(
@@ -152,20 +137,6 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void*
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
                      reinterpret_cast<uint64_t>(map)),
                  "r"(smem_u32(smem_src)), "r"(x), "r"(y)
-                 : "memory");
-}
-// 3-D variants: (x = element column, y = row inside the batch item, z = batch item).  Rows beyond the tensor's
-// extent are zero-filled on loads and dropped on stores, which is how ragged sequence lengths are handled.
-__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
-        : "memory");
-}
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* smem_src, int x, int y, int z) {
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
-                     reinterpret_cast<uint64_t>(map)),
-                 "r"(smem_u32(smem_src)), "r"(x), "r"(y), "r"(z)
                  : "memory");
 }
 // 4-D variants over a [batch, n, heads, d] tensor: (x = element inside the head, h = head, y = row, z = batch item).
@@ -228,12 +199,6 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr, uint32_t lbo_
 }
 // K-major operand tile [rows x 64] bf16, 128-byte swizzle: 8-row groups are 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc_kmajor(uint32_t saddr) { return umma_smem_desc(saddr, 16, 1024); }
-// MN-major operand made of [k_rows x 64] bf16 sub-tiles (128-byte swizzle): 8-row K groups are
-// 1024 bytes apart (stride offset); successive 64-element MN blocks are `mn_block_bytes` apart
-// (leading offset).
-__device__ __forceinline__ uint64_t umma_desc_mnmajor(uint32_t saddr, uint32_t mn_block_bytes) {
-    return umma_smem_desc(saddr, mn_block_bytes, 1024);
-}
 // Cheap descriptor arithmetic for the MMA-issuing thread.  The thread that issues tcgen05.mma is a
 // single lane; every instruction it spends per MMA delays the tensor pipe (a 128x128x16 MMA runs
 // for 64 cycles).  A descriptor is therefore split into its two 32-bit halves: the high half is a
