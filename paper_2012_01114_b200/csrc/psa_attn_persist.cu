@@ -81,6 +81,11 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
     constexpr bool SEP = Cfg::SEP_P;
     constexpr int VST = Cfg::VSTAGES;
     constexpr int KST = KVS ? Cfg::KSTAGES + Cfg::VSTAGES : Cfg::KSTAGES;     // stages of the K ring
+    // d = 128 with distinct K and V: V_j and K_{j+1} are needed by the same step of the issuing thread and released by
+    // it together, so they travel as one stage (K slot s and V slot s, one full and one empty barrier: v_full / v_empty):
+    // pair p of an item is (V_{p-1}, K_p), p = 0 .. blocks, the first without a V and the last without a K.  The
+    // issuing thread then probes one barrier and commits one release per key block instead of two of each.
+    constexpr bool PAIRED = !SEP && !KVS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;                                          // 2 tiles
@@ -151,42 +156,74 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                 const int nkv0 = kv_tiles(work.tile0, T, scheme);
                 const int nkv1 = work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0;
                 const int maxkv = max(nkv0, nkv1);
-                for (int j = 0; j < maxkv && ok; ++j) {
-                    {
-                        const int s = kc % KST;
-                        if (kc >= (uint32_t)KST) ok = mbar_wait(&bars.k_empty[s], ((kc / KST) - 1) & 1, abortp);
-                        if (!ok) break;
-                        mbar_arrive_expect_tx(&bars.k_full[s], Cfg::TILE_BYTES);
-                        for (int u = 0; u < Cfg::SUB; ++u)
-                            tma_load_4d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], 64 * u, h,
-                                        j * TILE, b);
-                        ++kc;
-                    }
-                    if (j == 0) {
-                        for (int t = 0; t < work.ntiles && ok; ++t) {
-                            if (qc[t] > 0) ok = mbar_wait(&bars.q_empty[t], (qc[t] - 1) & 1, abortp);
-                            if (!ok) break;
-                            mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
-                            for (int u = 0; u < Cfg::SUB; ++u)
-                                tma_load_4d(sQ + t * Cfg::TILE_BYTES + u * 16384, &maps.q, &bars.q_full[t],
-                                            64 * u, h, (work.tile0 + t) * TILE, b);
-                            ++qc[t];
-                        }
-                        if (!ok) break;
-                    }
-                    if constexpr (!KVS) {
+                if constexpr (PAIRED) {
+                    for (int p = 0; p <= maxkv && ok; ++p) {           // pair p = (V_{p-1}, K_p); vc counts pairs here
                         const int s = vc % VST;
                         if (vc >= (uint32_t)VST) ok = mbar_wait(&bars.v_empty[s], ((vc / VST) - 1) & 1, abortp);
                         if (!ok) break;
-                        mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
-                        for (int u = 0; u < Cfg::SUB; ++u)
-                            tma_load_4d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], 64 * u, h,
-                                        j * TILE, b);
+                        mbar_arrive_expect_tx(&bars.v_full[s], ((p > 0) + (p < maxkv)) * Cfg::TILE_BYTES);
+                        if (p < maxkv)
+                            for (int u = 0; u < Cfg::SUB; ++u)
+                                tma_load_4d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.v_full[s], 64 * u, h,
+                                            p * TILE, b);
+                        if (p > 0)
+                            for (int u = 0; u < Cfg::SUB; ++u)
+                                tma_load_4d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], 64 * u, h,
+                                            (p - 1) * TILE, b);
                         ++vc;
+                        if (p == 0) {
+                            for (int t = 0; t < work.ntiles && ok; ++t) {
+                                if (qc[t] > 0) ok = mbar_wait(&bars.q_empty[t], (qc[t] - 1) & 1, abortp);
+                                if (!ok) break;
+                                mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
+                                for (int u = 0; u < Cfg::SUB; ++u)
+                                    tma_load_4d(sQ + t * Cfg::TILE_BYTES + u * 16384, &maps.q, &bars.q_full[t],
+                                                64 * u, h, (work.tile0 + t) * TILE, b);
+                                ++qc[t];
+                            }
+                            if (!ok) break;
+                        }
+                        // the next item's index is fetched behind the item's first loads and long before it is needed
+                        if (p == 1) next = (int)gridDim.x + (int)atomicAdd(&dc->next_item, 1u);
                     }
-                    // the next item's index is fetched behind the item's first loads (the atomic's round trip of about
-                    // a thousand cycles would otherwise delay them) and long before it is needed
-                    if (j == 0) next = (int)gridDim.x + (int)atomicAdd(&dc->next_item, 1u);
+                } else {
+                    for (int j = 0; j < maxkv && ok; ++j) {
+                        {
+                            const int s = kc % KST;
+                            if (kc >= (uint32_t)KST) ok = mbar_wait(&bars.k_empty[s], ((kc / KST) - 1) & 1, abortp);
+                            if (!ok) break;
+                            mbar_arrive_expect_tx(&bars.k_full[s], Cfg::TILE_BYTES);
+                            for (int u = 0; u < Cfg::SUB; ++u)
+                                tma_load_4d(sK + s * Cfg::TILE_BYTES + u * 16384, &maps.k, &bars.k_full[s], 64 * u, h,
+                                            j * TILE, b);
+                            ++kc;
+                        }
+                        if (j == 0) {
+                            for (int t = 0; t < work.ntiles && ok; ++t) {
+                                if (qc[t] > 0) ok = mbar_wait(&bars.q_empty[t], (qc[t] - 1) & 1, abortp);
+                                if (!ok) break;
+                                mbar_arrive_expect_tx(&bars.q_full[t], Cfg::TILE_BYTES);
+                                for (int u = 0; u < Cfg::SUB; ++u)
+                                    tma_load_4d(sQ + t * Cfg::TILE_BYTES + u * 16384, &maps.q, &bars.q_full[t],
+                                                64 * u, h, (work.tile0 + t) * TILE, b);
+                                ++qc[t];
+                            }
+                            if (!ok) break;
+                        }
+                        if constexpr (!KVS) {
+                            const int s = vc % VST;
+                            if (vc >= (uint32_t)VST) ok = mbar_wait(&bars.v_empty[s], ((vc / VST) - 1) & 1, abortp);
+                            if (!ok) break;
+                            mbar_arrive_expect_tx(&bars.v_full[s], Cfg::TILE_BYTES);
+                            for (int u = 0; u < Cfg::SUB; ++u)
+                                tma_load_4d(sV + s * Cfg::TILE_BYTES + u * 16384, &maps.v, &bars.v_full[s], 64 * u, h,
+                                            j * TILE, b);
+                            ++vc;
+                        }
+                        // the next item's index is fetched behind the item's first loads (the atomic's round trip of about
+                        // a thousand cycles would otherwise delay them) and long before it is needed
+                        if (j == 0) next = (int)gridDim.x + (int)atomicAdd(&dc->next_item, 1u);
+                    }
                 }
                 idx = next;
             }
@@ -362,8 +399,10 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                                     work.ntiles > 1 ? kv_tiles(work.tile0 + 1, T, scheme) : 0};
                 const int maxkv = max(nkv[0], nkv[1]);
                 {
-                    // first scores of both tiles
-                    ok = mbar_wait(&bars.k_full[kbase % KST], (kbase / KST) & 1, abortp);
+                    // first scores of both tiles (PAIRED: kbase = vbase = the ring position of the item's pair 0, which
+                    // holds K_0 alone; pair j + 1 holds V_j and K_{j+1})
+                    if constexpr (PAIRED) ok = mbar_wait(&bars.v_full[vbase % VST], (vbase / VST) & 1, abortp);
+                    else ok = mbar_wait(&bars.k_full[kbase % KST], (kbase / KST) & 1, abortp);
                     for (int t = 0; t < work.ntiles && ok; ++t) {
                         ok = mbar_wait(&bars.q_full[t], parts[t] & 1, abortp);
                         if (!ok) break;
@@ -373,18 +412,20 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                         if (nkv[t] == 1) umma_commit(&bars.q_empty[t]);
                     }
                     if (!ok) break;
-                    if constexpr (!KVS) umma_commit(&bars.k_empty[kbase % KST]);
+                    if constexpr (PAIRED) umma_commit(&bars.v_empty[vbase % VST]);
+                    else if constexpr (!KVS) umma_commit(&bars.k_empty[kbase % KST]);
                     for (int j = 0; j < maxkv && ok; ++j) {
                         for (int t = 0; t < work.ntiles && ok; ++t) {
                             if (j >= nkv[t]) continue;
-                            const uint32_t vc = vbase + j, kc = kbase + j + 1;
+                            const uint32_t vc = vbase + j + (PAIRED ? 1 : 0), kc = kbase + j + 1;
                             const bool has_next = j + 1 < nkv[t];
                             // Operand tiles first.  A probe of a barrier costs this thread 150-200 cycles beside the
                             // busy softmax warps, so slot 1 does not repeat the ones slot 0 made for the same block.
                             if constexpr (!KVS)
                                 if (t == 0 || j >= nkv[0]) ok = mbar_wait(&bars.v_full[vc % VST], (vc / VST) & 1, abortp);
-                            if (ok && has_next && (t == 0 || j + 1 >= nkv[0]))
-                                ok = mbar_wait(&bars.k_full[kc % KST], (kc / KST) & 1, abortp);
+                            if constexpr (!PAIRED)
+                                if (ok && has_next && (t == 0 || j + 1 >= nkv[0]))
+                                    ok = mbar_wait(&bars.k_full[kc % KST], (kc / KST) & 1, abortp);
                             if (ok) ok = mbar_wait(&bars.p_ready[t], (blk0[t] + j) & 1, abortp);
                             if (!ok) break;
                             tc_fence_after();
@@ -395,15 +436,15 @@ attn_persist_kernel(const __grid_constant__ PMaps maps, const __grid_constant__ 
                             const bool last_v = t == work.ntiles - 1 || j >= nkv[t + 1];
                             if (last_v) umma_commit(KVS ? &bars.k_empty[(kbase + j) % KST] : &bars.v_empty[vc % VST]);
                             if (has_next) {
-                                if constexpr (!KVS)
+                                if constexpr (!KVS && !PAIRED)
                                     if (t == work.ntiles - 1 || j + 1 >= nkv[t + 1]) umma_commit(&bars.k_empty[kc % KST]);
                                 if (j + 1 == nkv[t] - 1) umma_commit(&bars.q_empty[t]);
                             }
                         }
                     }
                 }
-                kbase += maxkv;
-                vbase += maxkv;
+                kbase += maxkv + (PAIRED ? 1 : 0);
+                vbase += maxkv + (PAIRED ? 1 : 0);
                 for (int t = 0; t < work.ntiles; ++t) { ++parts[t]; blk0[t] += nkv[t]; }
             }
             const unsigned long long block_macs = (unsigned long long)TILE * TILE * D;
