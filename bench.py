@@ -45,7 +45,7 @@ L2_FLUSH_BYTES = 256 << 20
 # kernel it was measured on; once one of them changes the roofline reports traffic = null.
 NCU_TRAFFIC = {
     "sources": {
-        "psa_attn_persist.cu": "1545c1ceb149fdb1acc7efc46fadbd9f8291f9393da26d70c70aeb3031511551",
+        "psa_attn_persist.cu": "6faaea0a489bb7cad4f9e6d78e8ed96dd45b2f6e759c65f8d8539c5ae1166c96",
         "psa_softmax.cuh": "d6f464522774d5fa8e06d7bee0caa46cdbc57e830deef1f6ed5d2fd01c6dae71",
         "psa_sched.h": "f58d760c07067dcd12ea1f5d021072901f1247fc43730932f168d76ee1dd69aa",
         "psa_gemm.cu": "aa5a23d2e10a143ef90f2ed14bea1e072da286f79f0fd239b70736824174756c",
@@ -57,21 +57,21 @@ NCU_TRAFFIC = {
     },
     "traffic_bytes": {
         "c4": {
-            "attn": 594941696
+            "attn": 590732032
         },
         "c3": {
-            "attn": 38173440,
-            "proj": 16342272
+            "attn": 38193152,
+            "proj": 16174080
         },
         "c2": {
-            "attn": 19240192,
-            "proj": 9854464
+            "attn": 19239680,
+            "proj": 9854208
         },
         "c5-n256-full": {
-            "attn": 1045856768
+            "attn": 1046764800
         },
         "c5-n256-masked": {
-            "attn": 1046352896
+            "attn": 1049001984
         }
     }
 }
