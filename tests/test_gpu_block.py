@@ -28,6 +28,13 @@ def _proj_macs(B, H, n, D, d, scheme):
     return ((1 if scheme == oracle.SYMMETRIC else 3) + 1) * B * n * D * H * d
 
 
+@pytest.mark.parametrize("scheme", [oracle.FULL, oracle.MASKED])
+def test_block_bf16_with_wide_heads(scheme):
+    # heads of 256 columns run on the one-row-tile kernel between the two projection launches
+    test_block_bf16_matches_oracle(scheme, 2, 2, 300, 128, 256)
+    test_block_bf16_matches_oracle(scheme, 1, 1, 257, 64, 192)
+
+
 @pytest.mark.parametrize("scheme", [oracle.FULL, oracle.MASKED, oracle.SYMMETRIC])
 @pytest.mark.parametrize("B,H,n,D,d", [(1, 1, 128, 64, 64), (2, 3, 256, 192, 64), (1, 2, 384, 320, 128),
                                        (2, 2, 333, 128, 64), (1, 12, 512, 768, 64)])

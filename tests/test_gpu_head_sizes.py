@@ -134,3 +134,14 @@ def test_symmetric_scheme_stops_at_128_columns():
     with pytest.raises(binding.PsaError) as e:
         binding.psa_attention_core(q, None, None, oracle.SYMMETRIC)
     assert e.value.status == binding.ERR_UNSUPPORTED
+
+
+def test_wide_heads_with_one_tensor_for_keys_and_values():
+    B, H, n, d = 1, 2, 384, 256
+    vq, bq = inputs.tensor(37, 4, (B, n, H, d), 1.0, "bf16")
+    vk, bk = inputs.tensor(37, 5, (B, n, H, d), 1.0, "bf16")
+    k = _dev(bk)
+    out = binding.psa_attention_core(_dev(bq), k, k, oracle.MASKED)
+    ref, _ = oracle.attention_core(vq, vk, vk, oracle.MASKED)
+    err = np.abs(_f64(out) - ref)
+    assert (err <= TOL_BF16 + 2.0 ** -8 * np.abs(ref)).all(), err.max()
